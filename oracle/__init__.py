@@ -1,0 +1,191 @@
+"""CPU oracle for the broadcast-schedule computation -- TEST INFRASTRUCTURE.
+
+A ctypes front end for ``bcast_oracle.c`` (plain C, single-threaded, written
+from the paper; see that file's header).  Nothing in the CUDA library or its
+Python binding may import this package; only the tests, the smoke check and the
+benchmark's CPU-baseline leg do.  This package in turn imports nothing from the
+CUDA side.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bcast_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lock = threading.Lock()
+_lib = None
+
+PAD = -(2 ** 31)
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no optimisation tricks, no threads)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-Wall", "-Wextra", "-shared", "-fPIC",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            i32p = ctypes.POINTER(ctypes.c_int32)
+            i64p = ctypes.POINTER(ctypes.c_int64)
+            u64p = ctypes.POINTER(ctypes.c_uint64)
+            i64 = ctypes.c_int64
+            lib.oracle_q.argtypes = [i64]
+            lib.oracle_skips.argtypes = [i64, i64p]
+            lib.oracle_baseblock.argtypes = [i64, i64]
+            lib.oracle_recvschedule.argtypes = [i64, i64, i32p, i64p]
+            lib.oracle_sendschedule_def.argtypes = [i64, i64, i32p]
+            lib.oracle_sendschedule_alg6.argtypes = [i64, i64, i32p, i32p, u64p]
+            lib.oracle_schedule_table.argtypes = [i64, i64, i64, i64, i32p, i32p]
+            lib.oracle_round_k.argtypes = [ctypes.c_int, i64, i64]
+            lib.oracle_round_block.argtypes = [ctypes.c_int, i64, i64, i32p]
+            lib.oracle_round_block.restype = i64
+            lib.oracle_broadcast_rounds.argtypes = [ctypes.c_int, i64, i32p, i32p, i32p, i64p, i64p]
+            lib.oracle_checksum.argtypes = [i64, u64p]
+            lib.oracle_schedule_batch.argtypes = [i32p, i32p, i32p, i64, ctypes.c_int32,
+                                                  ctypes.c_int32, i32p, i32p]
+            _lib = lib
+    return _lib
+
+
+def _i32(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def _i64(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
+
+
+def q_of(p: int) -> int:
+    q = _load().oracle_q(p)
+    if q < 0:
+        raise ValueError("p must be >= 1")
+    return q
+
+
+def skips(p: int) -> np.ndarray:
+    """Algorithm 2: skip[0..q] as int64."""
+    q = q_of(p)
+    out = np.zeros(q + 1, dtype=np.int64)
+    _load().oracle_skips(p, _i64(out))
+    return out
+
+
+def baseblock(p: int, r: int) -> int:
+    b = _load().oracle_baseblock(p, r)
+    if b < 0:
+        raise ValueError("bad (p, r)")
+    return b
+
+
+def recvschedule(p: int, r: int, with_stats: bool = False):
+    """Algorithm 5 for virtual rank r; optionally the Lemma 5/6 counters."""
+    q = q_of(p)
+    out = np.zeros(max(q, 1), dtype=np.int32)
+    st = np.zeros(5, dtype=np.int64)
+    if _load().oracle_recvschedule(p, r, _i32(out), _i64(st)) < 0:
+        raise ValueError("bad (p, r)")
+    out = out[:q]
+    if with_stats:
+        return out, dict(calls=int(st[0]), iters=int(st[1]), retests=int(st[2]),
+                         retest_hits=int(st[3]), oob=int(st[4]))
+    return out
+
+
+def sendschedule(p: int, r: int) -> np.ndarray:
+    """Send schedule by definition (q receive schedules)."""
+    q = q_of(p)
+    out = np.zeros(max(q, 1), dtype=np.int32)
+    if _load().oracle_sendschedule_def(p, r, _i32(out)) < 0:
+        raise ValueError("bad (p, r)")
+    return out[:q]
+
+
+def sendschedule_alg6(p: int, r: int):
+    """Algorithm 6 (second routine): (row, violations, violation-round mask)."""
+    q = q_of(p)
+    out = np.zeros(max(q, 1), dtype=np.int32)
+    v = ctypes.c_int32(0)
+    m = ctypes.c_uint64(0)
+    if _load().oracle_sendschedule_alg6(p, r, _i32(out), ctypes.byref(v), ctypes.byref(m)) < 0:
+        raise ValueError("bad (p, r)")
+    return out[:q], int(v.value), int(m.value)
+
+
+def schedule_table(p: int, root: int = 0, rank_begin: int = 0, rank_end: int | None = None,
+                   want_recv: bool = True, want_send: bool = True):
+    """(recvblock, sendblock) int32 tables [rank_end-rank_begin, q] for actual ranks."""
+    if rank_end is None:
+        rank_end = p
+    q = q_of(p)
+    n = rank_end - rank_begin
+    recv = np.zeros((max(n, 0), q), dtype=np.int32) if want_recv else None
+    send = np.zeros((max(n, 0), q), dtype=np.int32) if want_send else None
+    rc = _load().oracle_schedule_table(p, root, rank_begin, rank_end,
+                                       _i32(recv) if want_recv else None,
+                                       _i32(send) if want_send else None)
+    if rc < 0:
+        raise ValueError("bad arguments to schedule_table (%d)" % rc)
+    return recv, send
+
+
+def round_k(q: int, n: int, j: int) -> int:
+    return _load().oracle_round_k(q, n, j)
+
+
+def round_block(q: int, n: int, j: int, row) -> int:
+    """Block moved in communication round j for a schedule row: -1 none, -2 bad args."""
+    row = np.ascontiguousarray(row, dtype=np.int32)
+    return int(_load().oracle_round_block(q, n, j, _i32(row)))
+
+
+def broadcast_rounds(q: int, n: int, recvrow, sendrow):
+    """Algorithm 1 as printed for one processor: (x, k[], raw recv[], raw send[])."""
+    recvrow = np.ascontiguousarray(recvrow, dtype=np.int32)
+    sendrow = np.ascontiguousarray(sendrow, dtype=np.int32)
+    rounds = n - 1 + q
+    k = np.zeros(rounds, dtype=np.int32)
+    rr = np.zeros(rounds, dtype=np.int64)
+    sr = np.zeros(rounds, dtype=np.int64)
+    x = _load().oracle_broadcast_rounds(q, n, _i32(recvrow), _i32(sendrow), _i32(k), _i64(rr), _i64(sr))
+    if x < 0:
+        raise ValueError("bad arguments")
+    return x, k, rr, sr
+
+
+def checksum(p: int) -> int:
+    """Order-independent 64-bit checksum of the full schedule of p (root 0)."""
+    c = ctypes.c_uint64(0)
+    if _load().oracle_checksum(p, ctypes.byref(c)) < 0:
+        raise ValueError("bad p")
+    return int(c.value)
+
+
+def schedule_batch(p, rank, root, row_stride: int = 31, pad: int = PAD,
+                   want_recv: bool = True, want_send: bool = True):
+    """Independent (p, rank, root) queries, rows padded to row_stride with pad."""
+    p = np.ascontiguousarray(p, dtype=np.int32)
+    rank = np.ascontiguousarray(rank, dtype=np.int32)
+    root = np.ascontiguousarray(root, dtype=np.int32)
+    nq = p.shape[0]
+    recv = np.zeros((nq, row_stride), dtype=np.int32) if want_recv else None
+    send = np.zeros((nq, row_stride), dtype=np.int32) if want_send else None
+    rc = _load().oracle_schedule_batch(_i32(p), _i32(rank), _i32(root), nq, row_stride, pad,
+                                       _i32(recv) if want_recv else None,
+                                       _i32(send) if want_send else None)
+    if rc < 0:
+        raise ValueError("bad query in batch")
+    return recv, send

@@ -1,0 +1,448 @@
+/*
+ * bcast_oracle.c -- TEST INFRASTRUCTURE, not product code.
+ *
+ * A plain, slow, single-threaded CPU statement of the round-optimal broadcast
+ * schedule of Traff, "Optimal Broadcast Schedules in Logarithmic Time ..."
+ * (arXiv 2407.18004).  It exists only so that the CUDA library can be compared
+ * with something written straight from the paper.  It shares no code, header,
+ * table or helper with the CUDA path and must never be linked into, imported
+ * by or called from it.  Only the tests, the smoke check and the benchmark's
+ * CPU-baseline leg use it.
+ *
+ * The receive schedule has no closed definition: it is whatever Algorithm 5
+ * (with Algorithms 2, 3 and 4) produces, so those are executed here step by
+ * step, with the paper's variable names, a real doubly linked list and real
+ * recursion.  The send schedule HAS a plain definition (Section 2.3:
+ * sendblock[k] of r is recvblock[k] of (r+skip[k]) mod p) and that definition
+ * is what the table functions use.  Algorithm 6 is kept as a second,
+ * independent routine (oracle_sendschedule_alg6) that the tests cross-check
+ * against the definition.
+ *
+ * Readings taken where the paper is silent (all listed in the design notes):
+ *  - Algorithm 4: r, r', s, e are passed by value; k is passed by value and
+ *    handed back as the return value; recvblock/next/prev are shared.
+ *  - Algorithm 4's recursive call passes the same e, so the callee tests it
+ *    once more.  Kept as printed.
+ *  - skip[k+1] is never needed with k = q; the oracle records it in `oob`
+ *    if that ever happens instead of reading past the array.
+ *  - p = 1 gives q = 0 and empty schedules; Algorithm 3's repeat-loop is not
+ *    entered then.
+ *  - all quantities are 64-bit: p+r, 2p and r'+skip[e] exceed 32 bits for
+ *    large p.
+ *
+ * Every function is pinned by the CPU tests against values the paper prints
+ * (Tables 1-3, the p=11 baseblock string), closed forms (powers of two), the
+ * four correctness conditions, the doubling observations and a brute-force
+ * broadcast simulation.  No function here is "parity unpinned".
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_MAXQ 64
+
+typedef struct {
+    int      q;
+    int64_t  p;
+    int64_t  skip[ORACLE_MAXQ + 2];
+    /* linked list over indices -1..q, stored with an offset of one */
+    int      next_[ORACLE_MAXQ + 3];
+    int      prev_[ORACLE_MAXQ + 3];
+    int      recvblock[ORACLE_MAXQ + 1];
+    /* instrumentation for the bounds the paper states (Lemmas 5 and 6) */
+    int64_t  calls;      /* recursive calls, the first invocation not counted */
+    int64_t  iters;      /* while-loop iterations over all calls              */
+    int64_t  retests;    /* iterations that are a callee's first look at the
+                            very index its caller just tested                 */
+    int64_t  retest_hits;/* how many of those passed the outer test           */
+    int64_t  oob;        /* skip[k+1] wanted with k >= q                      */
+} oracle_ctx;
+
+#define NEXT(c, e) ((c)->next_[(e) + 1])
+#define PREV(c, e) ((c)->prev_[(e) + 1])
+
+/* q = ceil(log2 p)  (Section 2, "we let p denote ... and take q = ...") */
+int oracle_q(int64_t p)
+{
+    int q = 0;
+    if (p < 1) return -1;
+    while (((int64_t)1 << q) < p) q++;
+    return q;
+}
+
+/* Algorithm 2: skips by repeated halving with rounding up. skip has q+1 slots. */
+int oracle_skips(int64_t p, int64_t *skip)
+{
+    int q = oracle_q(p);
+    int k;
+    if (q < 0) return -1;
+    k = q;
+    skip[k] = p;
+    while (k > 0) {
+        skip[k - 1] = skip[k] - skip[k] / 2;
+        k = k - 1;
+    }
+    return q;
+}
+
+/* Algorithm 3: smallest index of the canonical skip sequence of r; q for r=0. */
+static int baseblock_(const oracle_ctx *c, int64_t r)
+{
+    int k = c->q;
+    int64_t rp = 0;
+    if (c->q == 0) return c->q;
+    do {
+        k = k - 1;
+        if (rp + c->skip[k] == r) return k;
+        else if (rp + c->skip[k] < r) rp = rp + c->skip[k];
+    } while (k != 0);
+    return c->q;
+}
+
+/* Algorithm 4: greedy depth-first search with removal of accepted indices. */
+static int allblocks_(oracle_ctx *c, int64_t r, int64_t rp, int64_t s, int e, int k,
+                      int fresh_call)
+{
+    const int64_t *skip = c->skip;
+    int first = fresh_call;
+    while (e != -1) {
+        c->iters++;
+        if (first) c->retests++;
+        if (rp + skip[e] <= r - skip[k] && rp + skip[e] < s) {
+            if (first) c->retest_hits++;
+            if (k >= c->q) { c->oob++; return k; }
+            if (rp + skip[e] <= r - skip[k + 1]) {
+                c->calls++;
+                k = allblocks_(c, r, rp + skip[e], s, e, k, 1);
+            }
+            if (k >= c->q) { c->oob++; return k; }
+            if (rp > r - skip[k + 1]) return k;
+            s = rp + skip[e];
+            c->recvblock[k] = e;
+            k = k + 1;
+            NEXT(c, PREV(c, e)) = NEXT(c, e);
+            PREV(c, NEXT(c, e)) = PREV(c, e);
+        }
+        first = 0;
+        e = NEXT(c, e);
+    }
+    return k;
+}
+
+static int ctx_init_(oracle_ctx *c, int64_t p)
+{
+    memset(c, 0, sizeof(*c));
+    c->p = p;
+    c->q = oracle_skips(p, c->skip);
+    if (c->q < 0 || c->q > ORACLE_MAXQ) return -1;
+    return 0;
+}
+
+/* Algorithm 5: receive schedule of virtual rank r (root is rank 0). */
+static int recvschedule_(oracle_ctx *c, int64_t r, int *recvblock, int *b_out)
+{
+    int q = c->q, e, k, b;
+    for (e = 0; e <= q; e++) { NEXT(c, e) = e - 1; PREV(c, e) = e + 1; }
+    PREV(c, q) = -1; NEXT(c, -1) = q; PREV(c, -1) = 0;
+    b = baseblock_(c, r);
+    NEXT(c, PREV(c, b)) = NEXT(c, b);
+    PREV(c, NEXT(c, b)) = PREV(c, b);
+    k = allblocks_(c, c->p + r, 0, c->p + c->p, q, 0, 0);
+    for (k = 0; k < q; k++) {
+        if (c->recvblock[k] == q) recvblock[k] = b;
+        else recvblock[k] = c->recvblock[k] - q;
+    }
+    if (b_out) *b_out = b;
+    return 0;
+}
+
+int oracle_baseblock(int64_t p, int64_t r)
+{
+    oracle_ctx c;
+    if (ctx_init_(&c, p) || r < 0 || r >= p) return -1;
+    return baseblock_(&c, r);
+}
+
+/*
+ * Receive schedule of virtual rank r.  stats (may be NULL) receives
+ * {recursive calls, while iterations, re-test iterations, re-test hits, oob}.
+ */
+int oracle_recvschedule(int64_t p, int64_t r, int32_t *recvblock, int64_t *stats)
+{
+    oracle_ctx c;
+    int tmp[ORACLE_MAXQ + 1], k;
+    if (ctx_init_(&c, p) || r < 0 || r >= p) return -1;
+    /* poison so that an entry the search never wrote is seen by the tests */
+    for (k = 0; k <= c.q; k++) c.recvblock[k] = -1000;
+    recvschedule_(&c, r, tmp, NULL);
+    for (k = 0; k < c.q; k++) recvblock[k] = tmp[k];
+    if (stats) {
+        stats[0] = c.calls; stats[1] = c.iters; stats[2] = c.retests;
+        stats[3] = c.retest_hits; stats[4] = c.oob;
+    }
+    return c.q;
+}
+
+/* Send schedule by its definition: q receive schedules, one entry of each. */
+int oracle_sendschedule_def(int64_t p, int64_t r, int32_t *sendblock)
+{
+    oracle_ctx c;
+    int tmp[ORACLE_MAXQ + 1], k;
+    if (ctx_init_(&c, p) || r < 0 || r >= p) return -1;
+    for (k = 0; k < c.q; k++) {
+        int64_t t = (r + c.skip[k]) % p;
+        recvschedule_(&c, t, tmp, NULL);
+        sendblock[k] = tmp[k];
+    }
+    return c.q;
+}
+
+/*
+ * Algorithm 6, as a second routine that the tests compare with the definition.
+ * violations (may be NULL) receives the number of rounds that fell back to a
+ * receive-schedule computation; viol_mask (may be NULL) one bit per such round.
+ */
+int oracle_sendschedule_alg6(int64_t p, int64_t r, int32_t *sendblock,
+                             int32_t *violations, uint64_t *viol_mask)
+{
+    oracle_ctx c;
+    int q, k, b, nviol = 0;
+    int block[ORACLE_MAXQ + 1];
+    uint64_t vm = 0;
+    if (ctx_init_(&c, p) || r < 0 || r >= p) return -1;
+    q = c.q;
+    if (r == 0) {
+        for (k = 0; k < q; k++) sendblock[k] = k;
+    } else {
+        int64_t rp, e;
+        int cc;
+        b = baseblock_(&c, r);
+        rp = r; cc = b; e = p;
+        for (k = q - 1; k >= 1; k--) {
+            if (rp < c.skip[k]) {                       /* lower part */
+                if (rp + c.skip[k] < e || e < c.skip[k - 1] || (k == 1 && b > 0)) {
+                    sendblock[k] = cc;
+                } else {                                /* violation */
+                    recvschedule_(&c, (r + c.skip[k]) % p, block, NULL);
+                    sendblock[k] = block[k];
+                    nviol++; vm |= (uint64_t)1 << k;
+                }
+                if (e > c.skip[k]) e = c.skip[k];
+            } else {                                    /* upper part */
+                cc = k - q;
+                if (k == 1 || rp > c.skip[k] || e - c.skip[k] < c.skip[k - 1]) {
+                    sendblock[k] = cc;
+                } else if (rp + c.skip[k] > e) {        /* violation */
+                    recvschedule_(&c, (r + c.skip[k]) % p, block, NULL);
+                    sendblock[k] = block[k];
+                    nviol++; vm |= (uint64_t)1 << k;
+                } else {
+                    sendblock[k] = cc;
+                }
+                rp = rp - c.skip[k];
+                e = e - c.skip[k];
+            }
+        }
+        if (q > 0) sendblock[0] = b - q;
+    }
+    if (violations) *violations = nviol;
+    if (viol_mask) *viol_mask = vm;
+    return q;
+}
+
+/*
+ * Tables for actual ranks a in [rank_begin, rank_end) with the given root:
+ * row a-rank_begin holds the schedule of virtual rank (a-root+p) mod p
+ * (Section 2: a root other than 0 is handled by renumbering).  Either output
+ * may be NULL.  Row-major, q entries per row, no padding.
+ *
+ * Send rows follow the definition.  When the whole range [0,p) is asked for,
+ * the needed receive entries are already in this call's own receive table and
+ * are gathered from it; otherwise they are computed one receive schedule per
+ * entry.  The two routes are compared by the tests.
+ */
+int oracle_schedule_table(int64_t p, int64_t root, int64_t rank_begin, int64_t rank_end,
+                          int32_t *recv_out, int32_t *send_out)
+{
+    oracle_ctx c;
+    int tmp[ORACLE_MAXQ + 1], k, q;
+    int64_t a;
+    int32_t *recv_tab = recv_out;
+    int own = 0;
+    if (ctx_init_(&c, p)) return -1;
+    if (root < 0 || root >= p || rank_begin < 0 || rank_end > p || rank_begin > rank_end) return -1;
+    q = c.q;
+    if (q == 0) return 0;
+    {
+        int full = (rank_begin == 0 && rank_end == p);
+        if (full && send_out && !recv_tab) {
+            recv_tab = (int32_t *)malloc((size_t)p * q * sizeof(int32_t));
+            if (!recv_tab) return -2;
+            own = 1;
+        }
+        if (recv_tab) {
+            for (a = rank_begin; a < rank_end; a++) {
+                int64_t r = (a - root + p) % p;
+                recvschedule_(&c, r, tmp, NULL);
+                for (k = 0; k < q; k++) recv_tab[(a - rank_begin) * q + k] = tmp[k];
+            }
+        }
+        if (send_out) {
+            for (a = rank_begin; a < rank_end; a++) {
+                for (k = 0; k < q; k++) {
+                    if (full) {
+                        int64_t t = (a + c.skip[k]) % p;     /* actual to-processor */
+                        send_out[a * q + k] = recv_tab[t * q + k];
+                    } else {
+                        int64_t r = (a - root + p) % p;
+                        recvschedule_(&c, (r + c.skip[k]) % p, tmp, NULL);
+                        send_out[(a - rank_begin) * q + k] = tmp[k];
+                    }
+                }
+            }
+        }
+    }
+    if (own) free(recv_tab);
+    return q;
+}
+
+/*
+ * Algorithm 1, the part that turns a schedule row into the block of one round.
+ * n blocks, communication round j in [0, n-1+q): x = (q - (n-1) mod q) mod q
+ * virtual rounds precede it, so i = x + j, k = i mod q, and after the shift by
+ * -x (+q for i<x) and one +q per earlier use the entry reads
+ * sched[k] + q*floor(i/q) - x  (Theorem 1).  Negative: nothing is transferred
+ * (returns -1); above n-1: block n-1.
+ */
+int oracle_round_k(int q, int64_t n, int64_t j)
+{
+    int64_t x;
+    if (q < 1 || n < 1 || j < 0 || j >= n - 1 + q) return -1;
+    x = (q - (n - 1) % q) % q;
+    return (int)((x + j) % q);
+}
+
+int64_t oracle_round_block(int q, int64_t n, int64_t j, const int32_t *sched_row)
+{
+    int64_t x, i, raw;
+    int k;
+    if (q < 1 || n < 1 || j < 0 || j >= n - 1 + q) return -2;
+    x = (q - (n - 1) % q) % q;
+    i = x + j;
+    k = (int)(i % q);
+    /* the printed form: subtract x, add q when k < x, then q per earlier use */
+    raw = (int64_t)sched_row[k] - x;
+    if (k < x) raw += q;
+    {
+        /* uses of entry k before round i: rounds i' in [x, i) with i' mod q = k */
+        int64_t first = (k >= x) ? k : k + q;   /* first round >= x with residue k */
+        int64_t uses = (i - first) / q;
+        raw += uses * q;
+    }
+    if (raw < 0) return -1;
+    if (raw > n - 1) return n - 1;
+    return raw;
+}
+
+/*
+ * Algorithm 1 executed as printed, for one processor: shift both schedule rows
+ * by -x (+q for entries i < x), then walk rounds i = x .. n+q-1+x-1, reading
+ * entry k = i mod q and adding q to it after each use.  Outputs one value per
+ * communication round j = i - x: the round index k and the raw (uncapped,
+ * possibly negative) receive and send block numbers.  The caller applies the
+ * rules the paper leaves to the Send||Recv operation.
+ */
+int oracle_broadcast_rounds(int q, int64_t n, const int32_t *recvrow, const int32_t *sendrow,
+                            int32_t *k_out, int64_t *recv_raw, int64_t *send_raw)
+{
+    int64_t rb[ORACLE_MAXQ + 1], sb[ORACLE_MAXQ + 1];
+    int64_t x, i;
+    int k;
+    if (q < 1 || q > ORACLE_MAXQ || n < 1) return -1;
+    x = (q - (n - 1) % q) % q;
+    for (i = 0; i < q; i++) {
+        rb[i] = (int64_t)recvrow[i] - x;
+        sb[i] = (int64_t)sendrow[i] - x;
+        if (i < x) { rb[i] += q; sb[i] += q; }
+    }
+    for (i = x; i < n + q - 1 + x; i++) {
+        k = (int)(i % q);
+        k_out[i - x] = k;
+        recv_raw[i - x] = rb[k];
+        send_raw[i - x] = sb[k];
+        sb[k] += q;
+        rb[k] += q;
+    }
+    return (int)x;
+}
+
+/*
+ * Checksum of the whole schedule of p (root 0), used by the verification sweep:
+ * the wrapping 64-bit sum over all ranks r and rounds k of mix(key), with
+ *   key = r * 2^32 + k * 2^16 + (recv mod 256) * 2^8 + (send mod 256)
+ * and mix the finaliser of the SplitMix64 generator (Steele, Lea, Flood 2014):
+ *   z ^= z >> 30; z *= 0xbf58476d1ce4e5b9; z ^= z >> 27;
+ *   z *= 0x94d049bb133111eb; z ^= z >> 31.
+ * A sum, so that the order of evaluation does not matter.
+ */
+static uint64_t mix64_(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xbf58476d1ce4e5b9ULL;
+    z ^= z >> 27; z *= 0x94d049bb133111ebULL;
+    z ^= z >> 31;
+    return z;
+}
+
+int oracle_checksum(int64_t p, uint64_t *checksum)
+{
+    int q = oracle_q(p);
+    int32_t *recv, *send;
+    int64_t r;
+    int k;
+    uint64_t sum = 0;
+    if (q < 0) return -1;
+    if (q == 0) { *checksum = 0; return 0; }
+    recv = (int32_t *)malloc((size_t)p * q * sizeof(int32_t));
+    send = (int32_t *)malloc((size_t)p * q * sizeof(int32_t));
+    if (!recv || !send) { free(recv); free(send); return -2; }
+    oracle_schedule_table(p, 0, 0, p, recv, send);
+    for (r = 0; r < p; r++)
+        for (k = 0; k < q; k++) {
+            uint64_t key = ((uint64_t)r << 32) | ((uint64_t)k << 16)
+                         | ((uint64_t)(recv[r * q + k] & 0xff) << 8)
+                         | (uint64_t)(send[r * q + k] & 0xff);
+            sum += mix64_(key);
+        }
+    free(recv); free(send);
+    *checksum = sum;
+    return q;
+}
+
+/*
+ * Independent (p, rank, root) queries: row i of each output has row_stride
+ * entries; the first q_i hold the schedule of virtual rank
+ * (rank_i - root_i + p_i) mod p_i, the rest hold `pad`.
+ */
+int oracle_schedule_batch(const int32_t *p, const int32_t *rank, const int32_t *root,
+                          int64_t nq, int32_t row_stride, int32_t pad,
+                          int32_t *recv_out, int32_t *send_out)
+{
+    int64_t i;
+    int k;
+    for (i = 0; i < nq; i++) {
+        int64_t pi = p[i], r;
+        int q = oracle_q(pi);
+        if (q < 0 || q > row_stride || rank[i] < 0 || rank[i] >= pi || root[i] < 0 || root[i] >= pi)
+            return -1;
+        r = ((int64_t)rank[i] - root[i] + pi) % pi;
+        if (recv_out) {
+            oracle_recvschedule(pi, r, recv_out + i * row_stride, NULL);
+            for (k = q; k < row_stride; k++) recv_out[i * row_stride + k] = pad;
+        }
+        if (send_out) {
+            oracle_sendschedule_def(pi, r, send_out + i * row_stride);
+            for (k = q; k < row_stride; k++) send_out[i * row_stride + k] = pad;
+        }
+    }
+    return 0;
+}
