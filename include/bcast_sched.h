@@ -1,0 +1,165 @@
+/*
+ * bcast_sched.h -- C ABI of the broadcast-schedule library (CUDA, sm_100a).
+ *
+ * Computes, for p processors on the ceil(log2 p)-regular circulant graph, the
+ * round-optimal n-block broadcast schedule of J. L. Traff, "Optimal Broadcast
+ * Schedules in Logarithmic Time with Applications to Broadcast, All-Broadcast,
+ * Reduction and All-Reduction" (arXiv 2407.18004): the skips, and for each
+ * processor its recvblock[] and sendblock[] arrays of q = ceil(log2 p) entries.
+ *
+ * Conventions for every entry point
+ *  - Plain C types only.  "host" pointers are ordinary process memory; "device"
+ *    pointers are CUDA global memory of the current device.  The caller owns
+ *    every buffer; the library allocates nothing and keeps no state between
+ *    calls (it is thread-safe).
+ *  - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
+ *    Device work is enqueued on it and the call returns without synchronising.
+ *  - Return value: >= 0 on success (where stated, the value of q), otherwise a
+ *    negative BCAST_E* code.  Bad arguments are detected on the host before
+ *    anything is launched; nothing is thrown across the ABI.
+ *  - 1 <= p <= 2^31-1.  Processors are numbered 0..p-1.  A root other than 0 is
+ *    handled by renumbering (Section 2): the row of actual rank a holds the
+ *    schedule of virtual rank (a - root + p) mod p.
+ *  - Schedule entries are int32 in [-q, q-1] for rounds k = 0..q-1.  A negative
+ *    entry names a block of an earlier phase (Algorithm 1 adds q per phase).
+ */
+#ifndef BCAST_SCHED_H
+#define BCAST_SCHED_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BCAST_OK            0
+#define BCAST_EINVAL_P     -1   /* p < 1 or p > 2^31-1                                  */
+#define BCAST_EINVAL_ROOT  -2   /* root outside [0, p)                                  */
+#define BCAST_EINVAL_RANGE -3   /* not 0 <= rank_begin <= rank_end <= p, or p_lo > p_hi */
+#define BCAST_ENULL        -4   /* a required pointer is NULL                           */
+#define BCAST_EALIGN       -5   /* a device pointer is not aligned as documented        */
+#define BCAST_EINVAL_N     -6   /* n < 1, q < 1 or nq < 0                               */
+#define BCAST_EINVAL_ROUND -7   /* round j outside [0, n-1+q)                           */
+#define BCAST_ECUDA        -8   /* a CUDA runtime call failed (launch, attribute query) */
+#define BCAST_ESTRIDE      -9   /* row_stride below 31                                  */
+#define BCAST_ESCRATCH     -10  /* scratch buffer too small for a single p of the range */
+
+#define BCAST_NONE         (-1)         /* bcast_round_block: nothing moves in this round */
+#define BCAST_PAD          INT32_MIN    /* filler of unused row entries in the batch form */
+#define BCAST_MAX_Q        31
+
+/* Text for a BCAST_E* code (static storage, never NULL). */
+const char *bcast_strerror(int code);
+
+/*
+ * q = ceil(log2 p), the number of skips, of rounds per phase and of entries
+ * per schedule row (Section 2).  p = 1 gives 0.  Host only.
+ */
+int bcast_q(int32_t p);
+
+/*
+ * Algorithm 2: the skips of the circulant graph, skip[q] = p and
+ * skip[k-1] = ceil(skip[k] / 2), so skip[0] = 1 and skip[1] = 2 for p > 1.
+ * skip_host: host array of q+1 (at most 32) int32, written by the call.
+ * Returns q.  Host only, O(q).
+ */
+int bcast_skips(int32_t p, int32_t *skip_host);
+
+/*
+ * Algorithms 3-6 for every actual rank a in [rank_begin, rank_end):
+ * row a - rank_begin of recvblock_dev receives Algorithm 5's receive schedule
+ * and the same row of sendblock_dev the send schedule (Section 2.3:
+ * sendblock[k] of r equals recvblock[k] of (r + skip[k]) mod p) of virtual rank
+ * (a - root + p) mod p.
+ * Layout: device memory, int32, row-major, (rank_end - rank_begin) rows of
+ * exactly q entries, no padding; 4-byte aligned (16-byte aligned pointers take
+ * the vector-store path).  Either table pointer may be NULL to skip that table,
+ * not both.  An empty rank range and p = 1 (q = 0) succeed without a launch.
+ * Asynchronous on cuda_stream.  Returns q.
+ */
+int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
+                   int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);
+
+/*
+ * bcast_schedule with HOST output tables: the rank range is cut into chunks that
+ * fit the caller's device staging buffer (staging_dev, staging_bytes, 16-byte
+ * aligned; it must hold at least 32 rows of each requested table); each chunk
+ * is computed on the device and then copied into recvblock_host /
+ * sendblock_host (same layout as above, rows of the whole range) with
+ * cudaMemcpyAsync on cuda_stream.  Pinned host memory makes the copies
+ * asynchronous; pageable memory works and is slower.  The tables are complete
+ * once the stream has been synchronised.  Returns q, or BCAST_ESCRATCH when the
+ * staging buffer is too small.
+ */
+int bcast_schedule_host(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
+                        int32_t *recvblock_host, int32_t *sendblock_host,
+                        void *staging_dev, int64_t staging_bytes, void *cuda_stream);
+
+/*
+ * The same computation for nq independent queries (p_i, rank_i, root_i), all in
+ * device memory (int32, 4-byte aligned).  Row i of each output (int32,
+ * row-major, row_stride >= 31 entries per row) holds q_i = ceil(log2 p_i)
+ * schedule entries followed by BCAST_PAD up to row_stride.  A query with
+ * p_i < 1 or rank_i / root_i outside [0, p_i) gets a row of BCAST_PAD only and
+ * is counted in *bad_count_dev (device int32, may be NULL; the caller zeroes
+ * it).  Either output may be NULL, not both.  Asynchronous on cuda_stream.
+ */
+int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const int32_t *root_dev,
+                         int64_t nq, int32_t row_stride,
+                         int32_t *recvblock_dev, int32_t *sendblock_dev,
+                         int32_t *bad_count_dev, void *cuda_stream);
+
+/*
+ * Fused verification sweep (the exhaustive check of Section 2.3 / Appendix B)
+ * for every p in [p_lo, p_hi], root 0, all ranks, without writing tables to
+ * the caller: per p it computes all receive and send rows with the same
+ * device code as bcast_schedule, then checks on the device
+ *   [0] condition 1: recvblock[k]_r = sendblock[k] of (r - skip[k]) mod p
+ *   [1] condition 2: sendblock[k]_r = recvblock[k] of (r + skip[k]) mod p
+ *   [2] condition 3: the q received blocks are {-1..-q} \ {b-q} U {b}
+ *                    (the root: exactly {-1..-q})
+ *   [3] condition 4: sendblock[k] was received in a round j < k or is b - q
+ *   [4] Theorem 3:   more than 4 violations in Algorithm 6
+ *   [5] Lemmas 5, 6: more than q-1 descents or 2q+R list steps in the search
+ *   [6] root row sendblock[k] = k and sendblock[0] = b - q for the others
+ *   [7] internal:    the search ran into its iteration cap
+ * and adds the number of failing (rank, round) pairs to fail_counts_dev[0..7]
+ * (device uint32[8]; the caller zeroes it; all zero means every check passed).
+ * checksum_dev[p - p_lo] (device uint64, 8-byte aligned) receives the wrapping
+ * sum over all (r, k) of mix(r*2^32 + k*2^16 + (recv & 255)*2^8 + (send & 255)),
+ * mix being the SplitMix64 output finaliser; p = 1 gives 0.
+ * scratch_dev: device memory of scratch_bytes bytes, 16-byte aligned, used for
+ * the per-p tables while they are checked; bcast_verify_sweep_scratch_bytes()
+ * gives the size that lets every SM work; any size of at least
+ * 256 + (2 * q(p_hi) * p_hi rounded up to a multiple of 256) bytes is accepted
+ * and uses fewer blocks.  Contents after the call are unspecified.
+ * Asynchronous on cuda_stream; two sweeps that share a scratch buffer must not
+ * overlap on the device.
+ */
+int64_t bcast_verify_sweep_scratch_bytes(int32_t p_lo, int32_t p_hi);
+int bcast_verify_sweep(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
+                       uint32_t *fail_counts_dev, void *scratch_dev, int64_t scratch_bytes,
+                       void *cuda_stream);
+
+/*
+ * Algorithm 1's use of a schedule row, O(1) per round.  For n >= 1 blocks and
+ * communication round j in [0, n-1+q): x = (q - (n-1) mod q) mod q virtual
+ * rounds come first, so i = x + j, k = i mod q is the skip index of the round
+ * (peers (r +- skip[k]) mod p) and shift = q * floor(i/q) - x is what
+ * Theorem 1 adds to the row entry.  Host only.
+ */
+int bcast_round(int32_t q, int64_t n, int64_t j, int32_t *k_out, int64_t *shift_out);
+
+/*
+ * The block a processor moves in round j given its row (host, q entries):
+ * sched_row[k] + shift, capped to n-1, or BCAST_NONE when negative.  The rules
+ * "nothing is sent to the root" and "the root receives nothing" are the
+ * caller's.  Returns the block (>= 0), BCAST_NONE, or a BCAST_E* code (< -1).
+ */
+int64_t bcast_round_block(int32_t q, int64_t n, int64_t j, const int32_t *sched_row_host);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* BCAST_SCHED_H */

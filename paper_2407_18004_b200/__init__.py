@@ -1,0 +1,175 @@
+"""Python binding of the broadcast-schedule CUDA library (arXiv 2407.18004).
+
+A thin ctypes layer over ``libbcast_sched.so``: the functions carry the names of
+the C entry points in ``include/bcast_sched.h`` and only marshal arguments.
+PyTorch is used for device memory and streams; every step of the computation
+runs in the library's CUDA kernels.  There is no CPU fallback: if the library is
+missing it is built with nvcc, and if that fails the import error is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+
+from . import build as _build
+
+BCAST_NONE = -1
+BCAST_PAD = -(2 ** 31)
+BCAST_MAX_Q = 31
+
+_lib = None
+
+
+class BcastError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__("bcast_sched error %d: %s" % (code, bcast_strerror(code)))
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        lib = ctypes.CDLL(path)
+        i32, i64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+        lib.bcast_strerror.argtypes = [ctypes.c_int]
+        lib.bcast_strerror.restype = ctypes.c_char_p
+        lib.bcast_q.argtypes = [i32]
+        lib.bcast_skips.argtypes = [i32, vp]
+        lib.bcast_schedule.argtypes = [i32, i32, i64, i64, vp, vp, vp]
+        lib.bcast_schedule_host.argtypes = [i32, i32, i64, i64, vp, vp, vp, i64, vp]
+        lib.bcast_schedule_batch.argtypes = [vp, vp, vp, i64, i32, vp, vp, vp, vp]
+        lib.bcast_verify_sweep_scratch_bytes.argtypes = [i32, i32]
+        lib.bcast_verify_sweep_scratch_bytes.restype = i64
+        lib.bcast_verify_sweep.argtypes = [i32, i32, vp, vp, vp, i64, vp]
+        lib.bcast_round.argtypes = [i32, i64, i64, ctypes.POINTER(i32), ctypes.POINTER(i64)]
+        lib.bcast_round_block.argtypes = [i32, i64, i64, vp]
+        lib.bcast_round_block.restype = i64
+        _lib = lib
+    return _lib
+
+
+def library_path() -> str:
+    _load()
+    return _build.LIBRARY
+
+
+def _check(rc: int) -> int:
+    if rc < 0:
+        raise BcastError(int(rc))
+    return int(rc)
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor / numpy array, None -> NULL."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return getattr(stream, "cuda_stream", stream)
+
+
+# ------------------------------------------------------------------ host-only entry points
+def bcast_strerror(code: int) -> str:
+    return _load().bcast_strerror(code).decode()
+
+
+def bcast_q(p: int) -> int:
+    return _check(_load().bcast_q(p))
+
+
+def bcast_skips(p: int) -> np.ndarray:
+    q = bcast_q(p)
+    out = np.zeros(q + 1, dtype=np.int32)
+    _check(_load().bcast_skips(p, out.ctypes.data))
+    return out
+
+
+def bcast_round(q: int, n: int, j: int):
+    k = ctypes.c_int32(0)
+    shift = ctypes.c_int64(0)
+    _check(_load().bcast_round(q, n, j, ctypes.byref(k), ctypes.byref(shift)))
+    return int(k.value), int(shift.value)
+
+
+def bcast_round_block(q: int, n: int, j: int, sched_row) -> int:
+    row = np.ascontiguousarray(sched_row, dtype=np.int32)
+    rc = int(_load().bcast_round_block(q, n, j, row.ctypes.data))
+    if rc < BCAST_NONE:
+        raise BcastError(rc)
+    return rc
+
+
+# ------------------------------------------------------------------ device entry points
+def bcast_schedule(p: int, root: int, rank_begin: int, rank_end: int, recvblock, sendblock, stream=None) -> int:
+    """Fill int32 device tensors [rank_end-rank_begin, q]; either may be None. Returns q."""
+    return _check(_load().bcast_schedule(p, root, rank_begin, rank_end, _ptr(recvblock), _ptr(sendblock),
+                                         _stream(stream)))
+
+
+def bcast_schedule_host(p: int, root: int, rank_begin: int, rank_end: int, recvblock_host, sendblock_host,
+                        staging, stream=None) -> int:
+    """Host (ideally pinned) int32 output tables, filled chunk by chunk through a device staging tensor."""
+    nbytes = staging.numel() * staging.element_size()
+    return _check(_load().bcast_schedule_host(p, root, rank_begin, rank_end, _ptr(recvblock_host),
+                                              _ptr(sendblock_host), _ptr(staging), nbytes, _stream(stream)))
+
+
+def bcast_schedule_batch(p, rank, root, row_stride: int, recvblock, sendblock, bad_count=None, stream=None) -> int:
+    nq = p.numel()
+    return _check(_load().bcast_schedule_batch(_ptr(p), _ptr(rank), _ptr(root), nq, row_stride,
+                                               _ptr(recvblock), _ptr(sendblock), _ptr(bad_count), _stream(stream)))
+
+
+def bcast_verify_sweep_scratch_bytes(p_lo: int, p_hi: int) -> int:
+    return _check(_load().bcast_verify_sweep_scratch_bytes(p_lo, p_hi))
+
+
+def bcast_verify_sweep(p_lo: int, p_hi: int, checksum, fail_counts, scratch, stream=None) -> int:
+    nbytes = scratch.numel() * scratch.element_size()
+    return _check(_load().bcast_verify_sweep(p_lo, p_hi, _ptr(checksum), _ptr(fail_counts), _ptr(scratch),
+                                             nbytes, _stream(stream)))
+
+
+# ------------------------------------------------------------------ conveniences (allocation only)
+def schedule(p: int, root: int = 0, rank_begin: int = 0, rank_end: int | None = None, device="cuda",
+             want_recv: bool = True, want_send: bool = True):
+    """Allocate and fill (recvblock, sendblock) int32 device tensors for the rank range."""
+    import torch
+    if rank_end is None:
+        rank_end = p
+    q = bcast_q(p)
+    rows = max(rank_end - rank_begin, 0)
+    recv = torch.empty((rows, q), dtype=torch.int32, device=device) if want_recv else None
+    send = torch.empty((rows, q), dtype=torch.int32, device=device) if want_send else None
+    bcast_schedule(p, root, rank_begin, rank_end, recv, send)
+    return recv, send
+
+
+def schedule_batch(p, rank, root, row_stride: int = BCAST_MAX_Q):
+    """Allocate and fill padded rows for device int32 query tensors; returns (recv, send, bad_count)."""
+    import torch
+    nq = p.numel()
+    recv = torch.empty((nq, row_stride), dtype=torch.int32, device=p.device)
+    send = torch.empty((nq, row_stride), dtype=torch.int32, device=p.device)
+    bad = torch.zeros(1, dtype=torch.int32, device=p.device)
+    bcast_schedule_batch(p, rank, root, row_stride, recv, send, bad)
+    return recv, send, bad
+
+
+def verify_sweep(p_lo: int, p_hi: int, device="cuda"):
+    """Allocate buffers, run the fused verification sweep; returns (checksums uint64 as int64 tensor, fail_counts)."""
+    import torch
+    checksum = torch.zeros(p_hi - p_lo + 1, dtype=torch.int64, device=device)
+    fails = torch.zeros(8, dtype=torch.int32, device=device)
+    scratch = torch.empty(bcast_verify_sweep_scratch_bytes(p_lo, p_hi), dtype=torch.uint8, device=device)
+    bcast_verify_sweep(p_lo, p_hi, checksum, fails, scratch)
+    return checksum, fails

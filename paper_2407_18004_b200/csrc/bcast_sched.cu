@@ -1,0 +1,544 @@
+// C ABI and kernels of the broadcast-schedule library (see include/bcast_sched.h).
+//
+// Kernels
+//   schedule_table_kernel   one thread per rank, one warp per tile of 32 consecutive
+//                           ranks.  Each lane computes its receive row (Algorithms
+//                           3-5) and send row (Algorithm 6) in registers and drops the
+//                           entries as bytes into a per-warp shared-memory tile laid
+//                           out exactly like the output (row-major, q entries per row).
+//                           The warp then widens the tile to int32 and streams it out
+//                           as one contiguous run of 16-byte stores, so every store
+//                           instruction fills whole 32-byte sectors.  No block-wide
+//                           barrier: warps never wait for each other.
+//   schedule_batch_kernel   the same per-thread computation for independent
+//                           (p, rank, root) queries, rows padded to row_stride.
+//   verify_sweep_kernel     persistent blocks pull values of p from a queue, build the
+//                           tables of one p in scratch memory, then check the paper's
+//                           correctness conditions against them and reduce a checksum.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bcast_sched.h"
+#include "schedule_core.cuh"
+
+namespace bcast {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kThreads = kWarpsPerBlock * 32;
+constexpr int kMaxRowBytes = 32;                       // staged row: q <= 31 bytes (+ pad in batch form)
+
+// ------------------------------------------------------------------ per-rank rows
+// Where a thread puts entry k of a row: a byte row in shared memory ...
+struct ByteRow {
+    int8_t *row;
+    __device__ __forceinline__ void operator()(int k, int val) const { row[k] = (int8_t)val; }
+};
+// ... or one column element of a round-major table (entry k of rank r at base[k*stride]).
+struct StridedColumn {
+    int8_t *base;
+    size_t stride;
+    __device__ __forceinline__ void operator()(int k, int val) const { base[(size_t)k * stride] = (int8_t)val; }
+};
+
+// Both rows of virtual rank r.  Returns the number of Algorithm 6 violations.
+template <class Writer, class Stats>
+__device__ __forceinline__ int rank_rows(const Geometry &g, uint32_t r, Writer recv_row, Writer send_row,
+                                         bool want_recv, bool want_send, Stats &stats)
+{
+    const int q = g.q;
+    const int b = baseblock(g, r);
+    if (want_recv) recv_search(g, r, b, q - 1, recv_row, stats);
+    int nviol = 0;
+    if (want_send) {
+        if (r == 0u) {
+            for (int k = 0; k < q; ++k) send_row(k, k);
+        } else {
+            uint32_t viol = send_walk(g, r, b, send_row);
+            while (viol != 0u) {
+                const int k = 31 - __clz(viol);
+                viol ^= 1u << k;
+                uint32_t t = r + skip_of(g, k);
+                if (t >= g.p) t -= g.p;
+                NoStats ns;
+                send_row(k, recv_entry(g, t, k, ns));
+                ++nviol;
+            }
+        }
+    }
+    return nviol;
+}
+
+__device__ __forceinline__ int sext_byte(uint32_t w, uint32_t selector)
+{
+    int out;
+    // prmt: selector nibbles with bit 3 set replicate the sign of the chosen byte
+    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(out) : "r"(w), "r"(selector));
+    return out;
+}
+
+__device__ __forceinline__ int4 widen4(uint32_t w)
+{
+    int4 v;
+    v.x = sext_byte(w, 0x8880u);                       // byte 0 widened to int32
+    v.y = sext_byte(w, 0x9991u);
+    v.z = sext_byte(w, 0xAAA2u);
+    v.w = sext_byte(w, 0xBBB3u);
+    return v;
+}
+
+// Stream n_entries staged bytes out as int32, starting at out[0]; whole warp.
+__device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t *out, int n_entries,
+                                           bool vec_ok, int lane)
+{
+    const int8_t *stage_bytes = reinterpret_cast<const int8_t *>(stage_words);
+    int done = 0;
+    if (vec_ok) {
+        const int nvec = n_entries >> 2;
+        int4 *out4 = reinterpret_cast<int4 *>(out);
+        for (int i = lane; i < nvec; i += 32) __stcs(out4 + i, widen4(stage_words[i]));
+        done = nvec << 2;
+    }
+    for (int i = done + lane; i < n_entries; i += 32) __stcs(out + i, (int)stage_bytes[i]);
+}
+
+// ------------------------------------------------------------------ all ranks of one p
+__global__ void __launch_bounds__(kThreads)
+schedule_table_kernel(uint32_t p, uint32_t root, uint32_t rank_begin, uint32_t n_ranks,
+                      int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
+                      int recv_vec_ok, int send_vec_ok)
+{
+    __shared__ uint32_t stage[kWarpsPerBlock][2][kMaxRowBytes * 32 / 4];
+    const Geometry g = make_geometry(p);
+    const int q = g.q;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t n_tiles = (n_ranks + 31u) >> 5;
+    const uint32_t warps_total = gridDim.x * kWarpsPerBlock;
+    const ByteRow recv_row{reinterpret_cast<int8_t *>(stage[warp][0]) + lane * q};
+    const ByteRow send_row{reinterpret_cast<int8_t *>(stage[warp][1]) + lane * q};
+    const bool want_recv = recv_out != nullptr;
+    const bool want_send = send_out != nullptr;
+
+    for (uint32_t tile = blockIdx.x * kWarpsPerBlock + warp; tile < n_tiles; tile += warps_total) {
+        const uint32_t first = tile << 5;
+        const uint32_t idx = first + lane;
+        if (idx < n_ranks) {
+            const uint32_t a = rank_begin + idx;                          // actual rank
+            const uint32_t r = a >= root ? a - root : a + (p - root);     // virtual rank
+            NoStats ns;
+            rank_rows(g, r, recv_row, send_row, want_recv, want_send, ns);
+        }
+        __syncwarp();
+        const int rows = (int)min(32u, n_ranks - first);
+        const size_t base = (size_t)first * (size_t)q;
+        if (want_recv) flush_tile(stage[warp][0], recv_out + base, rows * q, recv_vec_ok, lane);
+        if (want_send) flush_tile(stage[warp][1], send_out + base, rows * q, send_vec_ok, lane);
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------ independent queries
+__global__ void __launch_bounds__(kThreads)
+schedule_batch_kernel(const int32_t *__restrict__ p_in, const int32_t *__restrict__ rank_in,
+                      const int32_t *__restrict__ root_in, int64_t nq, int row_stride,
+                      int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
+                      int32_t *bad_count, int recv_vec_ok, int send_vec_ok)
+{
+    // rows are staged 31 bytes wide and padded while they are written out
+    __shared__ uint32_t stage[kWarpsPerBlock][2][kMaxRowBytes * 32 / 4];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int64_t n_tiles = (nq + 31) >> 5;
+    const int64_t warps_total = (int64_t)gridDim.x * kWarpsPerBlock;
+    const ByteRow recv_row{reinterpret_cast<int8_t *>(stage[warp][0]) + lane * kMaxRowBytes};
+    const ByteRow send_row{reinterpret_cast<int8_t *>(stage[warp][1]) + lane * kMaxRowBytes};
+    const bool want_recv = recv_out != nullptr;
+    const bool want_send = send_out != nullptr;
+    constexpr int8_t kPadMark = -128;                  // no schedule entry is below -31
+
+    for (int64_t tile = (int64_t)blockIdx.x * kWarpsPerBlock + warp; tile < n_tiles; tile += warps_total) {
+        const int64_t first = tile << 5;
+        const int64_t idx = first + lane;
+        if (idx < nq) {
+            const int32_t pi = p_in[idx], ai = rank_in[idx], ri = root_in[idx];
+            int q = 0;
+            const bool ok = pi >= 1 && ai >= 0 && ai < pi && ri >= 0 && ri < pi;
+            if (!ok) {
+                if (bad_count) atomicAdd(bad_count, 1);
+            } else if (pi >= 2) {
+                const Geometry g = make_geometry((uint32_t)pi);
+                q = g.q;
+                const uint32_t a = (uint32_t)ai, root = (uint32_t)ri;
+                const uint32_t r = a >= root ? a - root : a + ((uint32_t)pi - root);
+                NoStats ns;
+                rank_rows(g, r, recv_row, send_row, want_recv, want_send, ns);
+            }
+            for (int k = q; k < kMaxRowBytes; ++k) { recv_row(k, kPadMark); send_row(k, kPadMark); }
+        }
+        __syncwarp();
+        const int rows = (int)min((int64_t)32, nq - first);
+        const int n_entries = rows * row_stride;
+        for (int t = 0; t < 2; ++t) {
+            int32_t *out = t == 0 ? recv_out : send_out;
+            if (out == nullptr) continue;
+            out += (size_t)first * (size_t)row_stride;
+            const int8_t *bytes = reinterpret_cast<const int8_t *>(stage[warp][t]);
+            const bool vec_ok = (t == 0 ? recv_vec_ok : send_vec_ok) && (row_stride & 3) == 0;
+            if (vec_ok) {
+                int4 *out4 = reinterpret_cast<int4 *>(out);
+                const int nvec = n_entries >> 2;
+                const int vec_per_row = row_stride >> 2;
+                for (int i = lane; i < nvec; i += 32) {
+                    const int row = i / vec_per_row;
+                    const int col = (i - row * vec_per_row) << 2;
+                    int e[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int cc = col + j;
+                        const int val = cc < kMaxRowBytes ? (int)bytes[row * kMaxRowBytes + cc] : (int)kPadMark;
+                        e[j] = val == (int)kPadMark ? BCAST_PAD : val;
+                    }
+                    __stcs(out4 + i, make_int4(e[0], e[1], e[2], e[3]));
+                }
+            } else {
+                for (int i = lane; i < n_entries; i += 32) {
+                    const int row = i / row_stride;
+                    const int cc = i - row * row_stride;
+                    const int val = cc < kMaxRowBytes ? (int)bytes[row * kMaxRowBytes + cc] : (int)kPadMark;
+                    __stcs(out + i, val == (int)kPadMark ? BCAST_PAD : val);
+                }
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------ verification sweep
+__device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xbf58476d1ce4e5b9ULL;
+    z ^= z >> 27; z *= 0x94d049bb133111ebULL;
+    z ^= z >> 31;
+    return z;
+}
+
+// Work queue: *queue_next counts values of p handed out, largest p first.
+__global__ void __launch_bounds__(kThreads)
+verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksum_out,
+                    uint32_t *__restrict__ fail_counts, int8_t *scratch,
+                    size_t scratch_per_block, unsigned int *queue_next)
+{
+    __shared__ uint32_t s_p;
+    __shared__ uint64_t s_sum[kWarpsPerBlock];
+    __shared__ uint32_t s_fail[8];
+    int8_t *tab = scratch + (size_t)blockIdx.x * scratch_per_block;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+
+    while (true) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned int ticket = atomicAdd(queue_next, 1u);
+            s_p = ticket <= p_hi - p_lo ? p_hi - ticket : 0u;
+        }
+        if (threadIdx.x < 8) s_fail[threadIdx.x] = 0u;
+        __syncthreads();
+        const uint32_t p = s_p;
+        if (p == 0u) break;
+        if (p == 1u) {
+            if (threadIdx.x == 0) checksum_out[p - p_lo] = 0ull;
+            continue;
+        }
+        const Geometry g = make_geometry(p);
+        const int q = g.q;
+        // tables of this p, round-major so that the checks read coalesced: tab[k*p + r]
+        int8_t *recv_tab = tab;
+        int8_t *send_tab = tab + (size_t)q * p;
+        uint32_t fail[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+
+        for (uint32_t r = threadIdx.x; r < p; r += kThreads) {
+            CountStats st;
+            const int nviol = rank_rows(g, r, StridedColumn{recv_tab + r, p}, StridedColumn{send_tab + r, p},
+                                        true, true, st);
+            if (nviol > 4) fail[4]++;
+            if (st.s.descents > q - 1 || st.s.steps > 2 * q + st.s.descents) fail[5]++;
+            if (st.s.capped) fail[7]++;
+        }
+        __syncthreads();
+
+        uint64_t sum = 0;
+        for (uint32_t r = threadIdx.x; r < p; r += kThreads) {
+            uint64_t seen = 0;                      // blocks received so far, bit (value + q)
+            int base = -1;                          // the non-negative received block
+            int first_send = 0;
+            for (int k = 0; k < q; ++k) {
+                const int rv = recv_tab[(size_t)k * p + r];
+                const int sv = send_tab[(size_t)k * p + r];
+                const uint32_t sk = skip_of(g, k);
+                const uint32_t f = r >= sk ? r - sk : r + (p - sk);
+                uint32_t t = r + sk; if (t >= p) t -= p;
+                if (rv != (int)send_tab[(size_t)k * p + f]) fail[0]++;
+                if (sv != (int)recv_tab[(size_t)k * p + t]) fail[1]++;
+                if (k == 0) first_send = sv;
+                if (r != 0u && k > 0) {
+                    // condition 4: sent block was received earlier, or is b - q (= sendblock[0])
+                    const bool held = ((seen >> (sv + q)) & 1ull) != 0ull || sv == first_send;
+                    if (!held) fail[3]++;
+                }
+                if (r == 0u && sv != k) fail[6]++;
+                if (rv >= 0) base = rv;
+                seen |= 1ull << (rv + q);
+                const uint64_t key = ((uint64_t)r << 32) | ((uint64_t)k << 16)
+                                   | ((uint64_t)(rv & 0xff) << 8) | (uint64_t)(sv & 0xff);
+                sum += mix64(key);
+            }
+            // condition 3 (and the root's row)
+            uint64_t want = (1ull << q) - 1ull;
+            if (r != 0u) {
+                if (base < 0) { fail[2]++; }
+                else {
+                    want = (want & ~(1ull << base)) | (1ull << (base + q));
+                    if (first_send != base - q) fail[6]++;
+                    if (base != baseblock(g, r)) fail[2]++;
+                }
+            }
+            if (seen != want) fail[2]++;
+        }
+        // block reduction of the checksum and the failure counters
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, off);
+        if (lane == 0) s_sum[warp] = sum;
+        for (int i = 0; i < 8; ++i)
+            if (fail[i] != 0u) atomicAdd(&s_fail[i], fail[i]);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint64_t total = 0;
+            for (int w = 0; w < kWarpsPerBlock; ++w) total += s_sum[w];
+            checksum_out[p - p_lo] = total;
+        }
+        if (threadIdx.x < 8 && s_fail[threadIdx.x] != 0u) atomicAdd(&fail_counts[threadIdx.x], s_fail[threadIdx.x]);
+    }
+}
+
+__global__ void zero_counter_kernel(unsigned int *c) { *c = 0u; }
+
+// ------------------------------------------------------------------ host helpers
+static int host_q(int64_t p)
+{
+    int q = 0;
+    while (((int64_t)1 << q) < p) ++q;
+    return q;
+}
+
+static int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    return sms;
+}
+
+static int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+static int64_t sweep_bytes_per_block(int32_t p_hi)
+{
+    return round_up((int64_t)2 * host_q(p_hi) * (int64_t)p_hi, 256);
+}
+
+constexpr int kSweepBlocksPerSm = 2;
+constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
+constexpr int kTableBlocksPerSm = 8;
+
+}  // namespace bcast
+
+using namespace bcast;
+
+extern "C" {
+
+const char *bcast_strerror(int code)
+{
+    switch (code) {
+    case BCAST_OK:            return "success";
+    case BCAST_EINVAL_P:      return "p must satisfy 1 <= p <= 2^31-1";
+    case BCAST_EINVAL_ROOT:   return "root must satisfy 0 <= root < p";
+    case BCAST_EINVAL_RANGE:  return "range must satisfy 0 <= begin <= end <= p (or p_lo <= p_hi)";
+    case BCAST_ENULL:         return "a required pointer is NULL";
+    case BCAST_EALIGN:        return "a device pointer is not aligned as documented";
+    case BCAST_EINVAL_N:      return "n, q and nq must be positive (nq may be 0)";
+    case BCAST_EINVAL_ROUND:  return "round j must satisfy 0 <= j < n-1+q";
+    case BCAST_ECUDA:         return "a CUDA runtime call failed";
+    case BCAST_ESTRIDE:       return "row_stride must be at least 31";
+    case BCAST_ESCRATCH:      return "scratch buffer too small";
+    default:                  return code > 0 ? "success" : "unknown error code";
+    }
+}
+
+int bcast_q(int32_t p)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    return host_q(p);
+}
+
+int bcast_skips(int32_t p, int32_t *skip_host)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (skip_host == nullptr) return BCAST_ENULL;
+    const int q = host_q(p);
+    int64_t s = p;
+    skip_host[q] = p;
+    for (int k = q; k > 0; --k) {
+        s = s - s / 2;
+        skip_host[k - 1] = (int32_t)s;
+    }
+    return q;
+}
+
+int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
+                   int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
+    if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
+    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
+    const int q = host_q(p);
+    const int64_t n_ranks = rank_end - rank_begin;
+    if (q == 0 || n_ranks == 0) return q;
+    const int sms = sm_count();
+    if (sms <= 0) return BCAST_ECUDA;
+    const int64_t n_tiles = (n_ranks + 31) / 32;
+    const int64_t blocks_needed = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int64_t grid_cap = (int64_t)sms * kTableBlocksPerSm;
+    const int grid = (int)(blocks_needed < grid_cap ? blocks_needed : grid_cap);
+    schedule_table_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
+        (uint32_t)p, (uint32_t)root, (uint32_t)rank_begin, (uint32_t)n_ranks, recvblock_dev, sendblock_dev,
+        ((uintptr_t)recvblock_dev & 15u) == 0, ((uintptr_t)sendblock_dev & 15u) == 0);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return q;
+}
+
+int bcast_schedule_host(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
+                        int32_t *recvblock_host, int32_t *sendblock_host,
+                        void *staging_dev, int64_t staging_bytes, void *cuda_stream)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
+    if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
+    if (recvblock_host == nullptr && sendblock_host == nullptr) return BCAST_ENULL;
+    if (staging_dev == nullptr) return BCAST_ENULL;
+    if ((uintptr_t)staging_dev & 15u) return BCAST_EALIGN;
+    const int q = host_q(p);
+    if (q == 0 || rank_end == rank_begin) return q;
+    const int n_tables = (recvblock_host != nullptr) + (sendblock_host != nullptr);
+    // ranks per chunk: a multiple of 32 so that every table slice stays 16-byte aligned
+    const int64_t row_bytes = (int64_t)q * 4;
+    int64_t chunk = staging_bytes / (row_bytes * n_tables) / 32 * 32;
+    if (chunk < 32) return BCAST_ESCRATCH;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    for (int64_t lo = rank_begin; lo < rank_end; lo += chunk) {
+        const int64_t hi = lo + chunk < rank_end ? lo + chunk : rank_end;
+        const int64_t rows = hi - lo;
+        int32_t *recv_dev = recvblock_host ? reinterpret_cast<int32_t *>(staging_dev) : nullptr;
+        int32_t *send_dev = sendblock_host
+            ? reinterpret_cast<int32_t *>(staging_dev) + (recvblock_host ? chunk * q : 0) : nullptr;
+        const int rc = bcast_schedule(p, root, lo, hi, recv_dev, send_dev, cuda_stream);
+        if (rc < 0) return rc;
+        const size_t off = (size_t)(lo - rank_begin) * q;
+        if (recvblock_host &&
+            cudaMemcpyAsync(recvblock_host + off, recv_dev, (size_t)rows * row_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+            return BCAST_ECUDA;
+        if (sendblock_host &&
+            cudaMemcpyAsync(sendblock_host + off, send_dev, (size_t)rows * row_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+            return BCAST_ECUDA;
+    }
+    return q;
+}
+
+int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const int32_t *root_dev,
+                         int64_t nq, int32_t row_stride,
+                         int32_t *recvblock_dev, int32_t *sendblock_dev,
+                         int32_t *bad_count_dev, void *cuda_stream)
+{
+    if (nq < 0) return BCAST_EINVAL_N;
+    if (row_stride < BCAST_MAX_Q) return BCAST_ESTRIDE;
+    if (p_dev == nullptr || rank_dev == nullptr || root_dev == nullptr) return BCAST_ENULL;
+    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)p_dev | (uintptr_t)rank_dev | (uintptr_t)root_dev | (uintptr_t)recvblock_dev |
+         (uintptr_t)sendblock_dev | (uintptr_t)bad_count_dev) & 3u) return BCAST_EALIGN;
+    if (nq == 0) return BCAST_OK;
+    const int sms = sm_count();
+    if (sms <= 0) return BCAST_ECUDA;
+    const int64_t n_tiles = (nq + 31) / 32;
+    const int64_t blocks_needed = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int64_t grid_cap = (int64_t)sms * kTableBlocksPerSm;
+    const int grid = (int)(blocks_needed < grid_cap ? blocks_needed : grid_cap);
+    schedule_batch_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
+        p_dev, rank_dev, root_dev, nq, row_stride, recvblock_dev, sendblock_dev, bad_count_dev,
+        ((uintptr_t)recvblock_dev & 15u) == 0, ((uintptr_t)sendblock_dev & 15u) == 0);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return BCAST_OK;
+}
+
+int64_t bcast_verify_sweep_scratch_bytes(int32_t p_lo, int32_t p_hi)
+{
+    if (p_lo < 1 || p_hi < 1) return BCAST_EINVAL_P;
+    if (p_lo > p_hi) return BCAST_EINVAL_RANGE;
+    const int sms = sm_count();
+    if (sms <= 0) return BCAST_ECUDA;
+    int64_t blocks = (int64_t)sms * kSweepBlocksPerSm;
+    const int64_t count = (int64_t)p_hi - p_lo + 1;
+    if (blocks > count) blocks = count;
+    return kSweepHeaderBytes + blocks * sweep_bytes_per_block(p_hi);
+}
+
+int bcast_verify_sweep(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
+                       uint32_t *fail_counts_dev, void *scratch_dev, int64_t scratch_bytes,
+                       void *cuda_stream)
+{
+    if (p_lo < 1 || p_hi < 1) return BCAST_EINVAL_P;
+    if (p_lo > p_hi) return BCAST_EINVAL_RANGE;
+    if (checksum_dev == nullptr || fail_counts_dev == nullptr || scratch_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)checksum_dev & 7u) || ((uintptr_t)fail_counts_dev & 3u) || ((uintptr_t)scratch_dev & 15u))
+        return BCAST_EALIGN;
+    const int64_t per_block = sweep_bytes_per_block(p_hi);
+    const int64_t usable = scratch_bytes - kSweepHeaderBytes;
+    if (usable < per_block) return BCAST_ESCRATCH;
+    const int sms = sm_count();
+    if (sms <= 0) return BCAST_ECUDA;
+    int64_t blocks = (int64_t)sms * kSweepBlocksPerSm;
+    const int64_t count = (int64_t)p_hi - p_lo + 1;
+    if (blocks > count) blocks = count;
+    if (blocks > usable / per_block) blocks = usable / per_block;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned int *queue = reinterpret_cast<unsigned int *>(scratch_dev);
+    zero_counter_kernel<<<1, 1, 0, stream>>>(queue);
+    verify_sweep_kernel<<<(int)blocks, kThreads, 0, stream>>>(
+        (uint32_t)p_lo, (uint32_t)p_hi, checksum_dev, fail_counts_dev,
+        reinterpret_cast<int8_t *>(scratch_dev) + kSweepHeaderBytes, (size_t)per_block, queue);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return BCAST_OK;
+}
+
+int bcast_round(int32_t q, int64_t n, int64_t j, int32_t *k_out, int64_t *shift_out)
+{
+    if (q < 1 || n < 1) return BCAST_EINVAL_N;
+    if (j < 0 || j >= n - 1 + q) return BCAST_EINVAL_ROUND;
+    const int64_t x = (q - (n - 1) % q) % q;
+    const int64_t i = x + j;
+    if (k_out) *k_out = (int32_t)(i % q);
+    if (shift_out) *shift_out = (i / q) * q - x;
+    return BCAST_OK;
+}
+
+int64_t bcast_round_block(int32_t q, int64_t n, int64_t j, const int32_t *sched_row_host)
+{
+    if (sched_row_host == nullptr) return BCAST_ENULL;
+    int32_t k = 0;
+    int64_t shift = 0;
+    const int rc = bcast_round(q, n, j, &k, &shift);
+    if (rc != BCAST_OK) return rc;
+    const int64_t raw = (int64_t)sched_row_host[k] + shift;
+    if (raw < 0) return BCAST_NONE;
+    return raw > n - 1 ? n - 1 : raw;
+}
+
+}  // extern "C"

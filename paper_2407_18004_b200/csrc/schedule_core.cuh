@@ -1,0 +1,191 @@
+// Per-rank schedule computation: Algorithms 2-6 of arXiv 2407.18004 restated for
+// one GPU thread per rank, all state in registers.
+//
+// What differs from the paper's sequential formulation (results are identical):
+//  * skip[k] is not stored: repeated ceil-halving composes to
+//    skip[k] = ((p-1) >> (q-k)) + 1, two ALU operations.
+//  * Algorithm 5's doubly linked list over the indices -1..q becomes a 32-bit set
+//    (q <= 31): "next smaller remaining index" is find-highest-set-bit below e,
+//    unlinking clears a bit.
+//  * Algorithm 4's recursion becomes a loop.  k and s behave as globals (k is
+//    returned by every call, and a caller never compares against s between a
+//    callee's return and its own next assignment to s), and the indices of the
+//    pending calls strictly decrease with depth, so the call stack is a second
+//    32-bit set and r' is the sum of its skips; "return" pops the lowest set bit.
+//    The callee's first test of the index its caller just used can never pass and
+//    is skipped.
+//  * Positions are kept as distances from the target R = p + r:
+//    u = R - r', v = R - s.  The tests of Algorithm 4 become
+//      r'+skip[e] <= R-skip[k]    <=>  skip[e] + skip[k]   <= u
+//      r'+skip[e] <  s            <=>  skip[e] + v         <  u
+//      r'+skip[e] <= R-skip[k+1]  <=>  skip[e] + skip[k+1] <= u
+//      r' > R-skip[k+1]           <=>  u < skip[k+1]
+//    and every quantity stays below 2^32 for p up to 2^31-1 (r'+skip[e] itself
+//    can reach 3p).  The initial s = 2p can never fail its test, so v starts at 0.
+#pragma once
+#include <stdint.h>
+
+namespace bcast {
+
+struct Geometry {
+    uint32_t p;     // number of processors, 2 <= p <= 2^31-1
+    uint32_t pm1;   // p - 1
+    int      q;     // ceil(log2 p), 1..31
+};
+
+__device__ __forceinline__ Geometry make_geometry(uint32_t p)
+{
+    Geometry g;
+    g.p = p;
+    g.pm1 = p - 1u;
+    g.q = 32 - __clz(p - 1u);          // p >= 2
+    return g;
+}
+
+// Algorithm 2 in closed form; valid for 0 <= k <= q.
+__device__ __forceinline__ uint32_t skip_of(const Geometry &g, int k)
+{
+    return (g.pm1 >> (g.q - k)) + 1u;
+}
+
+// Algorithm 3: smallest index of the canonical skip sequence of r; q for r = 0.
+__device__ __forceinline__ int baseblock(const Geometry &g, uint32_t r)
+{
+    uint32_t rem = r;                  // r - r'
+    for (int k = g.q - 1; k >= 0; --k) {
+        const uint32_t s = skip_of(g, k);
+        if (s == rem) return k;
+        if (s < rem) rem -= s;
+    }
+    return g.q;
+}
+
+// Counters the verification sweep reads; the table kernels pass a dummy.
+struct SearchStats {
+    int descents;       // recursive calls of Algorithm 4
+    int steps;          // list elements examined (Lemma 6 counts these)
+    int capped;         // the loop hit its safety cap
+};
+
+struct NoStats {
+    __device__ __forceinline__ void descent() {}
+    __device__ __forceinline__ void step() {}
+    __device__ __forceinline__ void cap() {}
+};
+
+struct CountStats {
+    SearchStats s{0, 0, 0};
+    __device__ __forceinline__ void descent() { s.descents++; }
+    __device__ __forceinline__ void step() { s.steps++; }
+    __device__ __forceinline__ void cap() { s.capped = 1; }
+};
+
+// Algorithms 4 and 5 for virtual rank r with baseblock b.  emit(k, value) is
+// called once for each k = 0..k_last in increasing order with the final schedule
+// value (b where the search accepted index q, else index - q).  k_last = q-1
+// yields the whole row; a smaller k_last stops early (used for one entry of
+// another rank's row).
+template <class Emit, class Stats>
+__device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b, int k_last,
+                                            Emit emit, Stats &stats)
+{
+    const int q = g.q;
+    uint32_t remaining = ((2u << q) - 1u) & ~(1u << b);   // list of skip indices, b unlinked
+    uint32_t pending = 0;                                 // indices of the calls in progress
+    uint32_t cand = remaining;                            // list part the current call still scans
+    uint32_t u = g.p + r;                                 // R - r'
+    uint32_t v = 0;                                       // R - s
+    int k = 0;
+    uint32_t sk_k = 1u;                                   // skip[k]
+    uint32_t sk_k1 = skip_of(g, 1);                       // skip[k+1]
+    uint32_t m = 1u;                                      // max(skip[k], v+1)
+    int guard = 6 * q + 16;                               // never reached; keeps the loop finite
+
+    while (true) {
+        if (--guard < 0) { stats.cap(); return; }
+        int e;
+        uint32_t bit, sk_e;
+        bool accept;
+        if (cand != 0u) {
+            e = 31 - __clz(cand);
+            bit = 1u << e;
+            cand ^= bit;
+            sk_e = skip_of(g, e);
+            stats.step();
+            // both outer tests of Algorithm 4: skip[e] <= u - max(skip[k], v+1)
+            if (u < m || sk_e > u - m) continue;
+            if (sk_e + sk_k1 <= u) {                      // room for a closer processor: descend
+                pending |= bit;
+                u -= sk_e;
+                stats.descent();
+                continue;
+            }
+            accept = (u >= sk_k1);
+            if (!accept) cand = 0u;                       // r' > R - skip[k+1]: return
+        } else {
+            if (pending == 0u) return;                    // outermost call ran off the list
+            bit = pending & (0u - pending);               // innermost pending call
+            pending ^= bit;
+            e = 31 - __clz(bit);
+            sk_e = skip_of(g, e);
+            u += sk_e;                                    // back in the caller's frame
+            accept = (u >= sk_k1);                        // else the caller returns as well
+        }
+        if (accept) {
+            emit(k, e == q ? b : e - q);
+            if (k == k_last) return;
+            v = u - sk_e;                                 // s = r' + skip[e]
+            remaining &= ~bit;
+            cand = remaining & (bit - 1u);
+            ++k;
+            sk_k = sk_k1;
+            sk_k1 = skip_of(g, k + 1 <= q ? k + 1 : q);
+            m = max(sk_k, v + 1u);
+        }
+    }
+}
+
+// Algorithm 6 for virtual rank r > 0 with baseblock b: emit(k, value) for
+// k = q-1..1 and then k = 0.  Rounds the fast rules cannot decide are returned as
+// a bit set (at most four by Theorem 3); the caller fills those entries with
+// recvblock[k] of rank (r + skip[k]) mod p.
+template <class Emit>
+__device__ __forceinline__ uint32_t send_walk(const Geometry &g, uint32_t r, int b, Emit emit)
+{
+    const int q = g.q;
+    uint32_t rp = r;            // virtual processor index r'
+    uint32_t e = g.p;           // upper bound on the range of virtual processors
+    int c = b;                  // block the lower part keeps sending
+    uint32_t violations = 0;
+    uint32_t sk = skip_of(g, q - 1);
+    for (int k = q - 1; k >= 1; --k) {
+        const uint32_t sk_below = skip_of(g, k - 1);
+        bool viol;
+        if (rp < sk) {                                    // lower part
+            viol = !(rp + sk < e || e < sk_below || (k == 1 && b > 0));
+            if (e > sk) e = sk;
+        } else {                                          // upper part
+            c = k - q;
+            viol = !(k == 1 || rp > sk || e - sk < sk_below) && (rp + sk > e);
+            rp -= sk;
+            e -= sk;
+        }
+        if (viol) violations |= 1u << k;
+        emit(k, c);
+        sk = sk_below;
+    }
+    emit(0, b - q);
+    return violations;
+}
+
+// One entry of another rank's receive schedule: recvblock[k] of virtual rank t.
+template <class Stats>
+__device__ __forceinline__ int recv_entry(const Geometry &g, uint32_t t, int k, Stats &stats)
+{
+    int value = 0;
+    const int bt = baseblock(g, t);
+    recv_search(g, t, bt, k, [&](int kk, int val) { if (kk == k) value = val; }, stats);
+    return value;
+}
+
+}  // namespace bcast

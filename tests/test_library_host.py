@@ -1,0 +1,106 @@
+"""CPU-side tests of the CUDA library: it loads, exports what the header declares,
+its host-only entry points agree with the oracle, and bad arguments are refused
+before anything is launched (no GPU needed for any of this)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2407_18004_b200 as bs
+from conftest import ROOT
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "bcast_sched.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bcast_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(bs.library_path())
+    names = declared_functions()
+    assert {"bcast_q", "bcast_skips", "bcast_schedule", "bcast_schedule_host", "bcast_schedule_batch",
+            "bcast_verify_sweep", "bcast_verify_sweep_scratch_bytes", "bcast_round", "bcast_round_block",
+            "bcast_strerror"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_q_and_skips_match_oracle():
+    rng = np.random.default_rng(7)
+    ps = list(range(1, 2000)) + [int(x) for x in rng.integers(2000, 2 ** 31 - 1, 2000)] + [2 ** 31 - 1, 2 ** 27 - 1]
+    for p in ps:
+        assert bs.bcast_q(p) == oracle.q_of(p)
+        assert bs.bcast_skips(p).tolist() == oracle.skips(p).tolist()
+
+
+def test_round_lookup_matches_oracle():
+    rng = np.random.default_rng(8)
+    for q in range(1, 12):
+        for n in list(range(1, 40)) + [1000, 12345]:
+            row = rng.integers(-q, q, q).astype(np.int32)
+            total = n - 1 + q
+            js = range(total) if total < 80 else [0, 1, q, total // 2, total - 2, total - 1]
+            for j in js:
+                k, shift = bs.bcast_round(q, n, j)
+                assert k == oracle.round_k(q, n, j)
+                assert bs.bcast_round_block(q, n, j, row) == oracle.round_block(q, n, j, row)
+                x = (q - (n - 1) % q) % q
+                assert shift == q * ((x + j) // q) - x
+
+
+def test_host_argument_errors():
+    assert bs.bcast_strerror(0) == "success"
+    for code in range(-10, 0):
+        assert bs.bcast_strerror(code) not in ("", "success")
+    with pytest.raises(bs.BcastError) as e:
+        bs.bcast_q(0)
+    assert e.value.code == -1
+    with pytest.raises(bs.BcastError) as e:
+        bs.bcast_round(0, 3, 0)
+    assert e.value.code == -6
+    with pytest.raises(bs.BcastError) as e:
+        bs.bcast_round(4, 3, 6)
+    assert e.value.code == -7
+    with pytest.raises(bs.BcastError) as e:
+        bs.bcast_round_block(4, 3, -1, [0, 0, 0, 0])
+    assert e.value.code == -7
+    lib = ctypes.CDLL(bs.library_path())
+    lib.bcast_schedule.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    fake = ctypes.c_void_p(0x1000)     # never dereferenced: every call below fails its checks first
+    assert lib.bcast_schedule(0, 0, 0, 0, fake, fake, None) == -1
+    assert lib.bcast_schedule(10, 10, 0, 10, fake, fake, None) == -2
+    assert lib.bcast_schedule(10, -1, 0, 10, fake, fake, None) == -2
+    assert lib.bcast_schedule(10, 0, 5, 4, fake, fake, None) == -3
+    assert lib.bcast_schedule(10, 0, 0, 11, fake, fake, None) == -3
+    assert lib.bcast_schedule(10, 0, 0, 10, None, None, None) == -4
+    assert lib.bcast_schedule(10, 0, 0, 10, ctypes.c_void_p(0x1002), None, None) == -5
+    assert lib.bcast_schedule(1, 0, 0, 1, fake, fake, None) == 0          # q = 0: nothing to launch
+    assert lib.bcast_schedule(10, 0, 3, 3, fake, fake, None) == 4         # empty range
+    lib.bcast_schedule_batch.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64, ctypes.c_int32] + [ctypes.c_void_p] * 4
+    assert lib.bcast_schedule_batch(fake, fake, fake, 5, 30, fake, fake, None, None) == -9
+    assert lib.bcast_schedule_batch(fake, fake, fake, -1, 31, fake, fake, None, None) == -6
+    assert lib.bcast_schedule_batch(None, fake, fake, 5, 31, fake, fake, None, None) == -4
+    assert lib.bcast_schedule_batch(fake, fake, fake, 5, 31, None, None, None, None) == -4
+    assert lib.bcast_schedule_batch(fake, fake, fake, 0, 31, fake, fake, None, None) == 0
+    lib.bcast_verify_sweep.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+    assert lib.bcast_verify_sweep(5, 4, fake, fake, fake, 1 << 20, None) == -3
+    assert lib.bcast_verify_sweep(0, 4, fake, fake, fake, 1 << 20, None) == -1
+    assert lib.bcast_verify_sweep(2, 4, None, fake, fake, 1 << 20, None) == -4
+    assert lib.bcast_verify_sweep(2, 1000, fake, fake, fake, 512, None) == -10
+
+
+def test_workload_generator_is_seeded_and_in_range():
+    from paper_2407_18004_b200 import workloads
+    p, rank, root = workloads.query_batch(10000, seed=0)
+    p2, rank2, root2 = workloads.query_batch(10000, seed=0)
+    assert np.array_equal(p, p2) and np.array_equal(rank, rank2) and np.array_equal(root, root2)
+    assert p.min() >= 2 and (rank >= 0).all() and (rank < p).all() and (root >= 0).all() and (root < p).all()
+    # log-uniform: every octave between 2^1 and 2^31 is populated
+    octave = np.floor(np.log2(p.astype(np.float64))).astype(int)
+    assert set(range(1, 31)) <= set(octave.tolist())
