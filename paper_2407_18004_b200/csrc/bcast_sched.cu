@@ -398,11 +398,11 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
     if (p < 1) return BCAST_EINVAL_P;
     if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
     if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
-    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
-    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
     const int q = host_q(p);
     const int64_t n_ranks = rank_end - rank_begin;
-    if (q == 0 || n_ranks == 0) return q;
+    if (q == 0 || n_ranks == 0) return q;              // zero-size tables: nothing to write
+    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
     const int sms = sm_count();
     if (sms <= 0) return BCAST_ECUDA;
     const int64_t n_tiles = (n_ranks + 31) / 32;
@@ -423,11 +423,11 @@ int bcast_schedule_host(int32_t p, int32_t root, int64_t rank_begin, int64_t ran
     if (p < 1) return BCAST_EINVAL_P;
     if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
     if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
+    const int q = host_q(p);
+    if (q == 0 || rank_end == rank_begin) return q;
     if (recvblock_host == nullptr && sendblock_host == nullptr) return BCAST_ENULL;
     if (staging_dev == nullptr) return BCAST_ENULL;
     if ((uintptr_t)staging_dev & 15u) return BCAST_EALIGN;
-    const int q = host_q(p);
-    if (q == 0 || rank_end == rank_begin) return q;
     const int n_tables = (recvblock_host != nullptr) + (sendblock_host != nullptr);
     // ranks per chunk: a multiple of 32 so that every table slice stays 16-byte aligned
     const int64_t row_bytes = (int64_t)q * 4;
