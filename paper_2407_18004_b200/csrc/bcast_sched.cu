@@ -20,6 +20,7 @@
 
 #include "../../include/bcast_sched.h"
 #include "schedule_core.cuh"
+#include "schedule_fast.cuh"
 
 namespace bcast {
 
@@ -32,12 +33,14 @@ constexpr int kMaxRowBytes = 32;                       // staged row: q <= 31 by
 struct ByteRow {
     int8_t *row;
     __device__ __forceinline__ void operator()(int k, int val) const { row[k] = (int8_t)val; }
+    __device__ __forceinline__ int get(int k) const { return row[k]; }
 };
 // ... or one column element of a round-major table (entry k of rank r at base[k*stride]).
 struct StridedColumn {
     int8_t *base;
     size_t stride;
     __device__ __forceinline__ void operator()(int k, int val) const { base[(size_t)k * stride] = (int8_t)val; }
+    __device__ __forceinline__ int get(int k) const { return base[(size_t)k * stride]; }
 };
 
 // Both rows of virtual rank r.  Returns the number of Algorithm 6 violations.
@@ -86,7 +89,9 @@ __device__ __forceinline__ int4 widen4(uint32_t w)
     return v;
 }
 
-// Stream n_entries staged bytes out as int32, starting at out[0]; whole warp.
+// Stream n_entries staged bytes out as int32, starting at out[0]; a group of kGroup
+// threads (a warp or the whole block), `lane` being the index within the group.
+template <int kGroup>
 __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t *out, int n_entries,
                                            bool vec_ok, int lane)
 {
@@ -95,45 +100,106 @@ __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t 
     if (vec_ok) {
         const int nvec = n_entries >> 2;
         int4 *out4 = reinterpret_cast<int4 *>(out);
-        for (int i = lane; i < nvec; i += 32) __stcs(out4 + i, widen4(stage_words[i]));
+        for (int i = lane; i < nvec; i += kGroup) __stcs(out4 + i, widen4(stage_words[i]));
         done = nvec << 2;
     }
-    for (int i = done + lane; i < n_entries; i += 32) __stcs(out + i, (int)stage_bytes[i]);
+    for (int i = done + lane; i < n_entries; i += kGroup) __stcs(out + i, (int)stage_bytes[i]);
 }
 
 // ------------------------------------------------------------------ all ranks of one p
+// An entry the closed-form pass could not decide: recvblock[k] of virtual rank `rank` is
+// wanted for every k in `mask` and goes to row `dest >> 1` of the receive (dest & 1 = 0)
+// or send (dest & 1 = 1) tile.
+struct SearchItem {
+    uint32_t rank;
+    uint32_t mask;
+    uint32_t dest;
+};
+
+constexpr int kItemsPerRank = 5;            // one receive item and at most four violations (Theorem 3)
+
+// Run the search for one queued item and drop the wanted entries into `row`.
+template <class Row, class Stats>
+__device__ __forceinline__ void resolve_item(const Geometry &g, const SearchItem &it, Row row, Stats &stats)
+{
+    const int b = baseblock(g, it.rank);
+    const uint32_t mask = it.mask;
+    recv_search(g, it.rank, b, 31 - __clz(mask),
+                [&](int k, int val) { if ((mask >> k) & 1u) row(k, val); }, stats);
+}
+
+// Rows of one rank through the closed forms; undecided entries are appended to the queue.
+template <int Q, class Row>
+__device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, const Geometry &g, uint32_t r,
+                                                    Row recv_row, Row send_row, uint32_t local_row,
+                                                    bool want_recv, bool want_send,
+                                                    SearchItem *queue, int *queue_count)
+{
+    uint32_t recv_flags, send_flags = 0;
+    if (r == 0u) {                                          // the root: sends block k in round k
+        for (int k = 0; k < Q; ++k) send_row(k, k);
+        recv_flags = (2u << (Q - 1)) - 1u;                  // its receive row comes from the search
+    } else {
+        recv_flags = closed_form_rows<Q>(tab, g.p, r, recv_row, send_row, &send_flags);
+    }
+    if (want_recv && recv_flags != 0u) {
+        const int slot = atomicAdd(queue_count, 1);
+        queue[slot] = SearchItem{r, recv_flags, local_row << 1};
+    }
+    uint32_t todo = want_send ? send_flags : 0u;
+    while (todo != 0u) {
+        const int k = 31 - __clz(todo);
+        todo ^= 1u << k;
+        uint32_t t = r + tab.skip[k];                       // the to-processor of round k
+        if (t >= g.p) t -= g.p;
+        const int slot = atomicAdd(queue_count, 1);
+        queue[slot] = SearchItem{t, 1u << k, (local_row << 1) | 1u};
+    }
+    return send_flags;
+}
+
+template <int Q>
 __global__ void __launch_bounds__(kThreads)
-schedule_table_kernel(uint32_t p, uint32_t root, uint32_t rank_begin, uint32_t n_ranks,
+schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t root,
+                      uint32_t rank_begin, uint32_t n_ranks,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
                       int recv_vec_ok, int send_vec_ok)
 {
-    __shared__ uint32_t stage[kWarpsPerBlock][2][kMaxRowBytes * 32 / 4];
+    // byte tiles laid out like the output: row-major, Q entries per rank, kThreads ranks
+    __shared__ uint32_t stage[2][kThreads * kMaxRowBytes / 4];
+    __shared__ SearchItem queue[kThreads * kItemsPerRank];
+    __shared__ int queue_count;
     const Geometry g = make_geometry(p);
-    const int q = g.q;
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const uint32_t n_tiles = (n_ranks + 31u) >> 5;
-    const uint32_t warps_total = gridDim.x * kWarpsPerBlock;
-    const ByteRow recv_row{reinterpret_cast<int8_t *>(stage[warp][0]) + lane * q};
-    const ByteRow send_row{reinterpret_cast<int8_t *>(stage[warp][1]) + lane * q};
+    const uint32_t n_tiles = (n_ranks + kThreads - 1u) / kThreads;
     const bool want_recv = recv_out != nullptr;
     const bool want_send = send_out != nullptr;
+    int8_t *recv_tile = reinterpret_cast<int8_t *>(stage[0]);
+    int8_t *send_tile = reinterpret_cast<int8_t *>(stage[1]);
 
-    for (uint32_t tile = blockIdx.x * kWarpsPerBlock + warp; tile < n_tiles; tile += warps_total) {
-        const uint32_t first = tile << 5;
-        const uint32_t idx = first + lane;
+    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        if (threadIdx.x == 0) queue_count = 0;
+        __syncthreads();                                   // also: the previous tile has been flushed
+        const uint32_t first = tile * kThreads;
+        const uint32_t idx = first + threadIdx.x;
         if (idx < n_ranks) {
             const uint32_t a = rank_begin + idx;                          // actual rank
             const uint32_t r = a >= root ? a - root : a + (p - root);     // virtual rank
-            NoStats ns;
-            rank_rows(g, r, recv_row, send_row, want_recv, want_send, ns);
+            rows_or_enqueue<Q>(tab, g, r, ByteRow{recv_tile + threadIdx.x * Q}, ByteRow{send_tile + threadIdx.x * Q},
+                               threadIdx.x, want_recv, want_send, queue, &queue_count);
         }
-        __syncwarp();
-        const int rows = (int)min(32u, n_ranks - first);
-        const size_t base = (size_t)first * (size_t)q;
-        if (want_recv) flush_tile(stage[warp][0], recv_out + base, rows * q, recv_vec_ok, lane);
-        if (want_send) flush_tile(stage[warp][1], send_out + base, rows * q, send_vec_ok, lane);
-        __syncwarp();
+        __syncthreads();
+        const int n_items = queue_count;
+        for (int i = threadIdx.x; i < n_items; i += kThreads) {
+            const SearchItem it = queue[i];
+            int8_t *tile_bytes = (it.dest & 1u) ? send_tile : recv_tile;
+            NoStats ns;
+            resolve_item(g, it, ByteRow{tile_bytes + (it.dest >> 1) * Q}, ns);
+        }
+        if (n_items > 0) __syncthreads();                  // n_items is the same for every thread
+        const int rows = (int)min((uint32_t)kThreads, n_ranks - first);
+        const size_t base = (size_t)first * (size_t)Q;
+        if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, rows * Q, recv_vec_ok, threadIdx.x);
+        if (want_send) flush_tile<kThreads>(stage[1], send_out + base, rows * Q, send_vec_ok, threadIdx.x);
     }
 }
 
@@ -222,6 +288,30 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z)
     return z;
 }
 
+// Level tables of p, built by the block itself (skip[] by Algorithm 2's closed form).
+__device__ __forceinline__ void fill_tables(LevelTables &tab, const Geometry &g)
+{
+    if (threadIdx.x == 0) {
+        uint32_t sum = 0;
+        for (int l = 0; l <= g.q; ++l) {
+            const uint32_t s = skip_of(g, l);
+            tab.skip[l] = s;
+            tab.below[l] = sum;
+            sum += s;
+        }
+        tab.below[g.q + 1] = sum;
+    }
+}
+
+template <int Q>
+__device__ __forceinline__ uint32_t sweep_rows(const LevelTables &tab, const Geometry &g, uint32_t r,
+                                               int8_t *recv_tab, int8_t *send_tab, uint32_t local_row,
+                                               SearchItem *queue, int *queue_count)
+{
+    return rows_or_enqueue<Q>(tab, g, r, StridedColumn{recv_tab + r, g.p}, StridedColumn{send_tab + r, g.p},
+                              local_row, true, true, queue, queue_count);
+}
+
 // Work queue: *queue_next counts values of p handed out, largest p first.
 __global__ void __launch_bounds__(kThreads)
 verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksum_out,
@@ -231,6 +321,9 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
     __shared__ uint32_t s_p;
     __shared__ uint64_t s_sum[kWarpsPerBlock];
     __shared__ uint32_t s_fail[8];
+    __shared__ LevelTables s_tab;
+    __shared__ SearchItem queue[kThreads * kItemsPerRank];
+    __shared__ int queue_count;
     int8_t *tab = scratch + (size_t)blockIdx.x * scratch_per_block;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -251,18 +344,41 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
         }
         const Geometry g = make_geometry(p);
         const int q = g.q;
+        fill_tables(s_tab, g);
         // tables of this p, round-major so that the checks read coalesced: tab[k*p + r]
         int8_t *recv_tab = tab;
         int8_t *send_tab = tab + (size_t)q * p;
         uint32_t fail[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
-        for (uint32_t r = threadIdx.x; r < p; r += kThreads) {
-            CountStats st;
-            const int nviol = rank_rows(g, r, StridedColumn{recv_tab + r, p}, StridedColumn{send_tab + r, p},
-                                        true, true, st);
-            if (nviol > 4) fail[4]++;
-            if (st.s.descents > q - 1 || st.s.steps > 2 * q + st.s.descents) fail[5]++;
-            if (st.s.capped) fail[7]++;
+        // the same closed-form pass and search queue as the table kernel, 256 ranks at a time
+        for (uint32_t first = 0; first < p; first += kThreads) {
+            if (threadIdx.x == 0) queue_count = 0;
+            __syncthreads();
+            const uint32_t r = first + threadIdx.x;
+            if (r < p) {
+                uint32_t viol = 0;
+                switch (q) {
+#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, r, recv_tab, send_tab, r, queue, &queue_count); break;
+                    BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
+                    BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
+                    BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
+                    BCAST_CASE(19) BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24)
+                    BCAST_CASE(25) BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30)
+                    BCAST_CASE(31)
+#undef BCAST_CASE
+                }
+                if (__popc(viol) > 4) fail[4]++;
+            }
+            __syncthreads();
+            const int n_items = queue_count;
+            for (int i = threadIdx.x; i < n_items; i += kThreads) {
+                const SearchItem it = queue[i];
+                int8_t *table = (it.dest & 1u) ? send_tab : recv_tab;
+                CountStats st;
+                resolve_item(g, it, StridedColumn{table + (it.dest >> 1), p}, st);
+                if (st.s.descents > q - 1 || st.s.steps > 2 * q + st.s.descents) fail[5]++;
+                if (st.s.capped) fail[7]++;
+            }
         }
         __syncthreads();
 
@@ -282,12 +398,12 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
                 if (k == 0) first_send = sv;
                 if (r != 0u && k > 0) {
                     // condition 4: sent block was received earlier, or is b - q (= sendblock[0])
-                    const bool held = ((seen >> (sv + q)) & 1ull) != 0ull || sv == first_send;
+                    const bool held = ((seen >> ((sv + q) & 63)) & 1ull) != 0ull || sv == first_send;
                     if (!held) fail[3]++;
                 }
                 if (r == 0u && sv != k) fail[6]++;
                 if (rv >= 0) base = rv;
-                seen |= 1ull << (rv + q);
+                seen |= 1ull << ((rv + q) & 63);
                 const uint64_t key = ((uint64_t)r << 32) | ((uint64_t)k << 16)
                                    | ((uint64_t)(rv & 0xff) << 8) | (uint64_t)(sv & 0xff);
                 sum += mix64(key);
@@ -337,6 +453,24 @@ static int sm_count()
     return sms;
 }
 
+static LevelTables host_tables(int64_t p, int q)
+{
+    LevelTables tab = {};
+    int64_t s = p;
+    tab.skip[q] = (uint32_t)p;
+    for (int k = q; k > 0; --k) {
+        s = s - s / 2;
+        tab.skip[k - 1] = (uint32_t)s;
+    }
+    uint32_t sum = 0;
+    for (int l = 0; l <= q; ++l) {
+        tab.below[l] = sum;
+        sum += tab.skip[l];
+    }
+    tab.below[q + 1] = sum;
+    return tab;
+}
+
 static int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
 static int64_t sweep_bytes_per_block(int32_t p_hi)
@@ -346,7 +480,7 @@ static int64_t sweep_bytes_per_block(int32_t p_hi)
 
 constexpr int kSweepBlocksPerSm = 2;
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
-constexpr int kTableBlocksPerSm = 8;
+constexpr int kTableBlocksPerSm = 6;
 
 }  // namespace bcast
 
@@ -405,13 +539,26 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
     if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
     const int sms = sm_count();
     if (sms <= 0) return BCAST_ECUDA;
-    const int64_t n_tiles = (n_ranks + 31) / 32;
-    const int64_t blocks_needed = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int64_t n_tiles = (n_ranks + kThreads - 1) / kThreads;
     const int64_t grid_cap = (int64_t)sms * kTableBlocksPerSm;
-    const int grid = (int)(blocks_needed < grid_cap ? blocks_needed : grid_cap);
-    schedule_table_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
-        (uint32_t)p, (uint32_t)root, (uint32_t)rank_begin, (uint32_t)n_ranks, recvblock_dev, sendblock_dev,
-        ((uintptr_t)recvblock_dev & 15u) == 0, ((uintptr_t)sendblock_dev & 15u) == 0);
+    const int grid = (int)(n_tiles < grid_cap ? n_tiles : grid_cap);
+    const LevelTables tab = host_tables(p, q);
+    const int recv_vec = ((uintptr_t)recvblock_dev & 15u) == 0, send_vec = ((uintptr_t)sendblock_dev & 15u) == 0;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    switch (q) {
+#define BCAST_CASE(N)                                                                                     \
+    case N:                                                                                               \
+        schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)root,         \
+            (uint32_t)rank_begin, (uint32_t)n_ranks, recvblock_dev, sendblock_dev, recv_vec, send_vec);   \
+        break;
+        BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6) BCAST_CASE(7)
+        BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12) BCAST_CASE(13)
+        BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18) BCAST_CASE(19)
+        BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24) BCAST_CASE(25)
+        BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30) BCAST_CASE(31)
+#undef BCAST_CASE
+    default: return BCAST_EINVAL_P;
+    }
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
 }
