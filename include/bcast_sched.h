@@ -131,7 +131,7 @@ int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const in
  * scratch_dev: device memory of scratch_bytes bytes, 16-byte aligned, used for
  * the per-p tables while they are checked; bcast_verify_sweep_scratch_bytes()
  * gives the size that lets every SM work; any size of at least
- * 256 + (2 * q(p_hi) * p_hi rounded up to a multiple of 256) bytes is accepted
+ * 256 + (2 * q(p_hi) * (p_hi + 1) rounded up to a multiple of 256) bytes is accepted
  * and uses fewer blocks.  Contents after the call are unspecified.
  * Asynchronous on cuda_stream; two sweeps that share a scratch buffer must not
  * overlap on the device.

@@ -129,18 +129,24 @@ __device__ __forceinline__ void resolve_item(const Geometry &g, const SearchItem
 }
 
 // Rows of one rank through the closed forms; undecided entries are appended to the queue.
+// Called by every lane of a warp (the closed-form pass votes across the warp): lanes
+// without a rank (`active` false) and the root compute the rows of rank 1 as a stand-in,
+// into the slot the caller gave them, and queue nothing for them.
 template <int Q, class Row>
 __device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, const Geometry &g, uint32_t r,
-                                                    Row recv_row, Row send_row, uint32_t local_row,
+                                                    bool active, Row recv_row, Row send_row, uint32_t local_row,
                                                     bool want_recv, bool want_send,
                                                     SearchItem *queue, int *queue_count)
 {
-    uint32_t recv_flags, send_flags = 0;
-    if (r == 0u) {                                          // the root: sends block k in round k
+    const bool is_root = r == 0u;
+    uint32_t send_flags = 0;
+    uint32_t recv_flags = closed_form_rows<Q>(tab, g.p, (active && !is_root) ? r : 1u, recv_row, send_row,
+                                              &send_flags);
+    if (!active) return 0u;
+    if (is_root) {                                          // the root sends block k in round k
         for (int k = 0; k < Q; ++k) send_row(k, k);
-        recv_flags = (2u << (Q - 1)) - 1u;                  // its receive row comes from the search
-    } else {
-        recv_flags = closed_form_rows<Q>(tab, g.p, r, recv_row, send_row, &send_flags);
+        recv_flags = (2u << (Q - 1)) - 1u;                  // and its receive row comes from the search
+        send_flags = 0u;
     }
     if (want_recv && recv_flags != 0u) {
         const int slot = atomicAdd(queue_count, 1);
@@ -181,11 +187,13 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         __syncthreads();                                   // also: the previous tile has been flushed
         const uint32_t first = tile * kThreads;
         const uint32_t idx = first + threadIdx.x;
-        if (idx < n_ranks) {
-            const uint32_t a = rank_begin + idx;                          // actual rank
+        {
+            const bool active = idx < n_ranks;
+            const uint32_t a = rank_begin + (active ? idx : 0u);          // actual rank
             const uint32_t r = a >= root ? a - root : a + (p - root);     // virtual rank
-            rows_or_enqueue<Q>(tab, g, r, ByteRow{recv_tile + threadIdx.x * Q}, ByteRow{send_tile + threadIdx.x * Q},
-                               threadIdx.x, want_recv, want_send, queue, &queue_count);
+            rows_or_enqueue<Q>(tab, g, r, active, ByteRow{recv_tile + threadIdx.x * Q},
+                               ByteRow{send_tile + threadIdx.x * Q}, threadIdx.x, want_recv, want_send,
+                               queue, &queue_count);
         }
         __syncthreads();
         const int n_items = queue_count;
@@ -303,13 +311,18 @@ __device__ __forceinline__ void fill_tables(LevelTables &tab, const Geometry &g)
     }
 }
 
+// The sweep keeps the tables of one p round-major with p + 1 slots per round: slot p
+// takes the stand-in rows of lanes beyond the last rank.
 template <int Q>
 __device__ __forceinline__ uint32_t sweep_rows(const LevelTables &tab, const Geometry &g, uint32_t r,
-                                               int8_t *recv_tab, int8_t *send_tab, uint32_t local_row,
+                                               int8_t *recv_tab, int8_t *send_tab,
                                                SearchItem *queue, int *queue_count)
 {
-    return rows_or_enqueue<Q>(tab, g, r, StridedColumn{recv_tab + r, g.p}, StridedColumn{send_tab + r, g.p},
-                              local_row, true, true, queue, queue_count);
+    const bool active = r < g.p;
+    const uint32_t slot = active ? r : g.p;
+    const size_t stride = (size_t)g.p + 1u;
+    return rows_or_enqueue<Q>(tab, g, active ? r : 1u, active, StridedColumn{recv_tab + slot, stride},
+                              StridedColumn{send_tab + slot, stride}, slot, true, true, queue, queue_count);
 }
 
 // Work queue: *queue_next counts values of p handed out, largest p first.
@@ -345,9 +358,10 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
         const Geometry g = make_geometry(p);
         const int q = g.q;
         fill_tables(s_tab, g);
-        // tables of this p, round-major so that the checks read coalesced: tab[k*p + r]
+        // tables of this p, round-major so that the checks read coalesced: tab[k*(p+1) + r]
+        const size_t stride = (size_t)p + 1u;
         int8_t *recv_tab = tab;
-        int8_t *send_tab = tab + (size_t)q * p;
+        int8_t *send_tab = tab + (size_t)q * stride;
         uint32_t fail[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
         // the same closed-form pass and search queue as the table kernel, 256 ranks at a time
@@ -355,10 +369,10 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
             if (threadIdx.x == 0) queue_count = 0;
             __syncthreads();
             const uint32_t r = first + threadIdx.x;
-            if (r < p) {
+            {
                 uint32_t viol = 0;
                 switch (q) {
-#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, r, recv_tab, send_tab, r, queue, &queue_count); break;
+#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, r, recv_tab, send_tab, queue, &queue_count); break;
                     BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
                     BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
                     BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
@@ -375,7 +389,7 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
                 const SearchItem it = queue[i];
                 int8_t *table = (it.dest & 1u) ? send_tab : recv_tab;
                 CountStats st;
-                resolve_item(g, it, StridedColumn{table + (it.dest >> 1), p}, st);
+                resolve_item(g, it, StridedColumn{table + (it.dest >> 1), stride}, st);
                 if (st.s.descents > q - 1 || st.s.steps > 2 * q + st.s.descents) fail[5]++;
                 if (st.s.capped) fail[7]++;
             }
@@ -388,13 +402,13 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
             int base = -1;                          // the non-negative received block
             int first_send = 0;
             for (int k = 0; k < q; ++k) {
-                const int rv = recv_tab[(size_t)k * p + r];
-                const int sv = send_tab[(size_t)k * p + r];
+                const int rv = recv_tab[(size_t)k * stride + r];
+                const int sv = send_tab[(size_t)k * stride + r];
                 const uint32_t sk = skip_of(g, k);
                 const uint32_t f = r >= sk ? r - sk : r + (p - sk);
                 uint32_t t = r + sk; if (t >= p) t -= p;
-                if (rv != (int)send_tab[(size_t)k * p + f]) fail[0]++;
-                if (sv != (int)recv_tab[(size_t)k * p + t]) fail[1]++;
+                if (rv != (int)send_tab[(size_t)k * stride + f]) fail[0]++;
+                if (sv != (int)recv_tab[(size_t)k * stride + t]) fail[1]++;
                 if (k == 0) first_send = sv;
                 if (r != 0u && k > 0) {
                     // condition 4: sent block was received earlier, or is b - q (= sendblock[0])
@@ -475,12 +489,12 @@ static int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
 static int64_t sweep_bytes_per_block(int32_t p_hi)
 {
-    return round_up((int64_t)2 * host_q(p_hi) * (int64_t)p_hi, 256);
+    return round_up((int64_t)2 * host_q(p_hi) * ((int64_t)p_hi + 1), 256);
 }
 
 constexpr int kSweepBlocksPerSm = 2;
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
-constexpr int kTableBlocksPerSm = 6;
+constexpr int kTableBlocksPerSm = 7;
 
 }  // namespace bcast
 

@@ -193,7 +193,7 @@ def test_verify_sweep_full_range():
 
 def test_verify_sweep_small_scratch_and_offsets():
     lo, hi = 1000, 1100
-    need = 256 + -(-2 * bs.bcast_q(hi) * hi // 256) * 256
+    need = 256 + -(-2 * bs.bcast_q(hi) * (hi + 1) // 256) * 256
     checksum = torch.zeros(hi - lo + 1, dtype=torch.int64, device="cuda")
     fails = torch.zeros(8, dtype=torch.int32, device="cuda")
     scratch = torch.empty(need, dtype=torch.uint8, device="cuda")       # room for one block only
