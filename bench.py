@@ -52,6 +52,32 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+def kernel_source_hash() -> str:
+    """sha256 over the CUDA sources: a recorded DRAM-traffic figure is only quoted for the kernel it was taken on."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2407_18004_b200", "csrc", "*"))):
+        with open(path, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(kernel: str, p: int):
+    """dram read+write bytes per launch from profiles/dram_traffic.txt, or None when the sources changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    sha = kernel_source_hash()
+    with open(path) as fh:
+        for line in fh:
+            parts = line.split()
+            if len(parts) >= 5 and not line.startswith("#") and parts[0] == kernel and parts[1] == str(p) \
+                    and parts[2] == sha:
+                return int(parts[3]) + int(parts[4])
+    return None
+
+
 class ClockSampler:
     """nvidia-smi clock/throttle samples while the timed region runs."""
 
@@ -271,11 +297,7 @@ def run_ours(args):
     peak, peak_src = measured_peaks()
     kernel_ms = statistics.mean(per_step_ms)
     achieved = table_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = None
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_path):
-        with open(traffic_path) as fh:
-            traffic = json.load(fh).get("schedule_table_kernel:" + args.workload)
+    traffic = recorded_traffic("schedule_table_kernel", p)
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
