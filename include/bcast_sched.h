@@ -43,10 +43,14 @@ extern "C" {
 #define BCAST_ECUDA        -8   /* a CUDA runtime call failed (launch, attribute query) */
 #define BCAST_ESTRIDE      -9   /* row_stride below 31                                  */
 #define BCAST_ESCRATCH     -10  /* scratch buffer too small for a single p of the range */
+#define BCAST_ETOOBIG      -11  /* p_hi above BCAST_STATIC_SWEEP_MAX_P                  */
 
 #define BCAST_NONE         (-1)         /* bcast_round_block: nothing moves in this round */
 #define BCAST_PAD          INT32_MIN    /* filler of unused row entries in the batch form */
 #define BCAST_MAX_Q        31
+
+#define BCAST_STATIC_SWEEP_BYTES  (8u << 20)   /* built-in scratch of bcast_verify_sweep_static */
+#define BCAST_STATIC_SWEEP_MAX_P  65536        /* largest p_hi it accepts                       */
 
 /* Text for a BCAST_E* code (static storage, never NULL). */
 const char *bcast_strerror(int code);
@@ -140,6 +144,39 @@ int64_t bcast_verify_sweep_scratch_bytes(int32_t p_lo, int32_t p_hi);
 int bcast_verify_sweep(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
                        uint32_t *fail_counts_dev, void *scratch_dev, int64_t scratch_bytes,
                        void *cuda_stream);
+
+/*
+ * bcast_verify_sweep for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this is a packaging variant of the sweep above.)
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they
+ * want a sweep: code running inside a memory-pool or real-time section that
+ * forbids allocation, a plug-in that is handed output buffers but no allocator,
+ * a process whose allocator is owned by another runtime.  For them the per-p
+ * tables go into a fixed array of BCAST_STATIC_SWEEP_BYTES (8 MiB) that is part
+ * of the library's device image; each GPU that loads the library holds it until
+ * the process ends.  The caller still owns and passes checksum_dev and
+ * fail_counts_dev (same meaning, alignment and zeroing rules as above).
+ *
+ * Limits and rules
+ *  - p_hi <= BCAST_STATIC_SWEEP_MAX_P (65536), else BCAST_ETOOBIG; nothing is
+ *    launched.  The array holds three blocks' worth of tables at that size, so
+ *    large ranges run with less parallelism than bcast_verify_sweep with the
+ *    scratch size it recommends; results are identical.
+ *  - The call itself performs no cudaMalloc/cudaFree and uses no allocating
+ *    library routine.
+ *  - The first call on each device looks the array's device address up
+ *    (cudaGetSymbolAddress, with that device current) and remembers it; make
+ *    that first call before any stream capture is started.
+ *  - All calls on a device share the one array and it keeps whatever the last
+ *    call left; the sweep clears its work-queue counter itself at the start of
+ *    each call and reads nothing else before writing it.  Two calls whose device
+ *    work overlaps (different streams, different host threads) race on the
+ *    array: serialise them.
+ * Asynchronous on cuda_stream.  Returns BCAST_OK or a BCAST_E* code.
+ */
+int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
+                              uint32_t *fail_counts_dev, void *cuda_stream);
 
 /*
  * Algorithm 1's use of a schedule row, O(1) per round.  For n >= 1 blocks and

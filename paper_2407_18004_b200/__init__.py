@@ -17,6 +17,7 @@ from . import build as _build
 BCAST_NONE = -1
 BCAST_PAD = -(2 ** 31)
 BCAST_MAX_Q = 31
+BCAST_STATIC_SWEEP_MAX_P = 65536
 
 _lib = None
 
@@ -43,6 +44,7 @@ def _load():
         lib.bcast_verify_sweep_scratch_bytes.argtypes = [i32, i32]
         lib.bcast_verify_sweep_scratch_bytes.restype = i64
         lib.bcast_verify_sweep.argtypes = [i32, i32, vp, vp, vp, i64, vp]
+        lib.bcast_verify_sweep_static.argtypes = [i32, i32, vp, vp, vp]
         lib.bcast_round.argtypes = [i32, i64, i64, ctypes.POINTER(i32), ctypes.POINTER(i64)]
         lib.bcast_round_block.argtypes = [i32, i64, i64, vp]
         lib.bcast_round_block.restype = i64
@@ -137,6 +139,16 @@ def bcast_verify_sweep(p_lo: int, p_hi: int, checksum, fail_counts, scratch, str
     nbytes = scratch.numel() * scratch.element_size()
     return _check(_load().bcast_verify_sweep(p_lo, p_hi, _ptr(checksum), _ptr(fail_counts), _ptr(scratch),
                                              nbytes, _stream(stream)))
+
+
+def bcast_verify_sweep_static(p_lo: int, p_hi: int, checksum, fail_counts, stream=None) -> int:
+    """The sweep for callers that may not allocate: its tables live in an 8 MiB array inside the library.
+
+    checksum / fail_counts are the caller's device tensors as for bcast_verify_sweep; p_hi <= 65536.
+    Calls share the array, so calls that could overlap on the device must be serialised.
+    """
+    return _check(_load().bcast_verify_sweep_static(p_lo, p_hi, _ptr(checksum), _ptr(fail_counts),
+                                                    _stream(stream)))
 
 
 # ------------------------------------------------------------------ conveniences (allocation only)

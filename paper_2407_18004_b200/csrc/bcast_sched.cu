@@ -18,6 +18,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/bcast_sched.h"
 #include "schedule_core.cuh"
 #include "schedule_fast.cuh"
@@ -516,6 +518,7 @@ const char *bcast_strerror(int code)
     case BCAST_ECUDA:         return "a CUDA runtime call failed";
     case BCAST_ESTRIDE:       return "row_stride must be at least 31";
     case BCAST_ESCRATCH:      return "scratch buffer too small";
+    case BCAST_ETOOBIG:       return "p_hi exceeds what the built-in scratch of bcast_verify_sweep_static holds";
     default:                  return code > 0 ? "success" : "unknown error code";
     }
 }
@@ -700,6 +703,40 @@ int64_t bcast_round_block(int32_t q, int64_t n, int64_t j, const int32_t *sched_
     const int64_t raw = (int64_t)sched_row_host[k] + shift;
     if (raw < 0) return BCAST_NONE;
     return raw > n - 1 ? n - 1 : raw;
+}
+
+// ------------------------------------------------------------------ sweep without caller scratch
+// The tables of the sweep live in this array instead of in memory the caller allocated.
+// It is part of the loaded module: every device that loads the library carries these
+// bytes until the process exits, which is why the size is kept modest.
+static __device__ __align__(256) unsigned char g_sweep_static_scratch[BCAST_STATIC_SWEEP_BYTES];
+
+// Device address of the array, looked up once per device.  In host code the array's
+// name is only a handle for the runtime, never an address a kernel may be given.
+static void *g_sweep_static_ptr[64];
+static std::mutex g_sweep_static_mutex;
+
+int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
+                              uint32_t *fail_counts_dev, void *cuda_stream)
+{
+    if (p_lo < 1 || p_hi < 1) return BCAST_EINVAL_P;
+    if (p_lo > p_hi) return BCAST_EINVAL_RANGE;
+    if (p_hi > BCAST_STATIC_SWEEP_MAX_P) return BCAST_ETOOBIG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BCAST_ECUDA;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_sweep_static_mutex);
+        if (g_sweep_static_ptr[dev] == nullptr) {
+            void *addr = nullptr;
+            if (cudaGetSymbolAddress(&addr, g_sweep_static_scratch) != cudaSuccess || addr == nullptr)
+                return BCAST_ECUDA;
+            g_sweep_static_ptr[dev] = addr;
+        }
+        scratch = g_sweep_static_ptr[dev];
+    }
+    return bcast_verify_sweep(p_lo, p_hi, checksum_dev, fail_counts_dev, scratch,
+                              (int64_t)BCAST_STATIC_SWEEP_BYTES, cuda_stream);
 }
 
 }  // extern "C"
