@@ -109,62 +109,134 @@ __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t 
 }
 
 // ------------------------------------------------------------------ all ranks of one p
-// An entry the closed-form pass could not decide: recvblock[k] of virtual rank `rank` is
-// wanted for every k in `mask` and goes to row `dest >> 1` of the receive (dest & 1 = 0)
-// or send (dest & 1 = 1) tile.
+// Work the closed-form pass leaves behind, collected per tile of kThreads consecutive ranks.
+//
+// SearchItem: recvblock[k] of virtual rank `rank` is wanted for every k in `mask` and goes
+// to row `row` of the tile's receive (table = 0) or send (table = 1) rows; base is the
+// rank's baseblock + 1 when the pass already knows it, else 0.
+// A copy (packed into 32 bits) says: sendblock[k] of row dst is recvblock[k] of row src of
+// the same tile (Section 2.3's definition, the to-processor being src), to be taken once
+// the searches of the tile are done.
 struct SearchItem {
     uint32_t rank;
     uint32_t mask;
-    uint32_t dest;
+    uint16_t row;
+    uint8_t table;
+    uint8_t base;
 };
 
-constexpr int kItemsPerRank = 5;            // one receive item and at most four violations (Theorem 3)
+constexpr int kSearchCapacity = 2 * kThreads;
+constexpr int kCopyCapacity = 2 * kThreads;
 
-// Run the search for one queued item and drop the wanted entries into `row`.
+struct TileQueue {
+    SearchItem search[kSearchCapacity];
+    uint32_t copy[kCopyCapacity];               // src | dst << 9 | k << 18
+    int n_search;
+    int n_copy;
+};
+
+// Run the search for one item and drop the wanted entries into `row`.
 template <class Row, class Stats>
 __device__ __forceinline__ void resolve_item(const Geometry &g, const SearchItem &it, Row row, Stats &stats)
 {
-    const int b = baseblock(g, it.rank);
+    const int b = it.base != 0 ? (int)it.base - 1 : baseblock(g, it.rank);
     const uint32_t mask = it.mask;
     recv_search(g, it.rank, b, 31 - __clz(mask),
                 [&](int k, int val) { if ((mask >> k) & 1u) row(k, val); }, stats);
 }
 
-// Rows of one rank through the closed forms; undecided entries are appended to the queue.
-// Called by every lane of a warp (the closed-form pass votes across the warp): lanes
-// without a rank (`active` false) and the root compute the rows of rank 1 as a stand-in,
-// into the slot the caller gave them, and queue nothing for them.
-template <int Q, class Row>
+// Queue a search; when the queue is full the calling thread does it on the spot.
+template <class Tile, class Stats>
+__device__ __forceinline__ void push_search(const Geometry &g, TileQueue &queue, const SearchItem &it,
+                                            const Tile &tile, Stats &stats)
+{
+    const int slot = atomicAdd(&queue.n_search, 1);
+    if (slot < kSearchCapacity) {
+        queue.search[slot] = it;
+    } else if (it.table == 0) {
+        resolve_item(g, it, tile.recv_row(it.row), stats);
+    } else {
+        resolve_item(g, it, tile.send_row(it.row), stats);
+    }
+}
+
+// Rows of one rank through the closed forms; what the pass cannot decide is queued.
+// Called by every lane of a warp: lanes without a rank (`active` false) and the root
+// compute the rows of rank 1 as a stand-in, into their own row of the tile, and queue
+// nothing for them.  `index` is the rank's row in the tile, `rows` the tile's row count;
+// consecutive rows hold consecutive virtual ranks (mod p).  Returns Algorithm 6's violations.
+template <int Q, class Tile, class Stats>
 __device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, const Geometry &g, uint32_t r,
-                                                    bool active, Row recv_row, Row send_row, uint32_t local_row,
-                                                    bool want_recv, bool want_send,
-                                                    SearchItem *queue, int *queue_count)
+                                                    bool active, const Tile &tile, uint32_t index, uint32_t rows,
+                                                    bool want_recv, bool want_send, TileQueue &queue, Stats &stats)
 {
     const bool is_root = r == 0u;
     uint32_t send_flags = 0;
+    int b = 0;
+    auto recv_row = tile.recv_row(index);
+    auto send_row = tile.send_row(index);
     uint32_t recv_flags = closed_form_rows<Q>(tab, g.p, (active && !is_root) ? r : 1u, recv_row, send_row,
-                                              &send_flags);
+                                              &send_flags, &b);
     if (!active) return 0u;
     if (is_root) {                                          // the root sends block k in round k
         for (int k = 0; k < Q; ++k) send_row(k, k);
         recv_flags = (2u << (Q - 1)) - 1u;                  // and its receive row comes from the search
         send_flags = 0u;
+        b = Q;
     }
-    if (want_recv && recv_flags != 0u) {
-        const int slot = atomicAdd(queue_count, 1);
-        queue[slot] = SearchItem{r, recv_flags, local_row << 1};
-    }
+    if (want_recv && recv_flags != 0u)
+        push_search(g, queue, SearchItem{r, recv_flags, (uint16_t)index, 0, (uint8_t)(b + 1)}, tile, stats);
     uint32_t todo = want_send ? send_flags : 0u;
     while (todo != 0u) {
         const int k = 31 - __clz(todo);
         todo ^= 1u << k;
-        uint32_t t = r + tab.skip[k];                       // the to-processor of round k
+        const uint32_t sk = tab.skip[k];
+        // the to-processor of round k: a row of this tile whose receive entry will be final
+        // after the tile's searches, or a rank that needs a search of its own
+        if (want_recv && index + sk < rows) {
+            const int slot = atomicAdd(&queue.n_copy, 1);
+            if (slot < kCopyCapacity) {
+                queue.copy[slot] = (index + sk) | (index << 9) | ((uint32_t)k << 18);
+                continue;
+            }
+        }
+        uint32_t t = r + sk;
         if (t >= g.p) t -= g.p;
-        const int slot = atomicAdd(queue_count, 1);
-        queue[slot] = SearchItem{t, 1u << k, (local_row << 1) | 1u};
+        push_search(g, queue, SearchItem{t, 1u << k, (uint16_t)index, 1, 0}, tile, stats);
     }
     return send_flags;
 }
+
+// After the closed-form pass of a tile and a barrier: searches, then (after another
+// barrier, only if needed) the copies.  Every thread of the block calls this.
+template <class Tile, class Stats>
+__device__ __forceinline__ void drain_queue(const Geometry &g, TileQueue &queue, const Tile &tile, Stats &stats)
+{
+    const int n_search = min(queue.n_search, kSearchCapacity);
+    const int n_copy = min(queue.n_copy, kCopyCapacity);
+    for (int i = threadIdx.x; i < n_search; i += kThreads) {
+        const SearchItem it = queue.search[i];
+        if (it.table == 0) resolve_item(g, it, tile.recv_row(it.row), stats);
+        else resolve_item(g, it, tile.send_row(it.row), stats);
+    }
+    if (n_copy > 0) {
+        __syncthreads();                                   // n_copy is the same for every thread
+        for (int i = threadIdx.x; i < n_copy; i += kThreads) {
+            const uint32_t c = queue.copy[i];
+            const int k = (int)(c >> 18);
+            tile.send_row((c >> 9) & 511u)(k, tile.recv_row(c & 511u).get(k));
+        }
+    }
+}
+
+// The table kernel's tile: byte rows in shared memory, laid out like the output.
+template <int Q>
+struct SharedTile {
+    int8_t *recv;
+    int8_t *send;
+    __device__ __forceinline__ ByteRow recv_row(uint32_t i) const { return ByteRow{recv + i * Q}; }
+    __device__ __forceinline__ ByteRow send_row(uint32_t i) const { return ByteRow{send + i * Q}; }
+};
 
 template <int Q>
 __global__ void __launch_bounds__(kThreads)
@@ -173,43 +245,34 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
                       int recv_vec_ok, int send_vec_ok)
 {
-    // byte tiles laid out like the output: row-major, Q entries per rank, kThreads ranks
     __shared__ uint32_t stage[2][kThreads * kMaxRowBytes / 4];
-    __shared__ SearchItem queue[kThreads * kItemsPerRank];
-    __shared__ int queue_count;
+    __shared__ TileQueue queue;
     const Geometry g = make_geometry(p);
     const uint32_t n_tiles = (n_ranks + kThreads - 1u) / kThreads;
     const bool want_recv = recv_out != nullptr;
     const bool want_send = send_out != nullptr;
-    int8_t *recv_tile = reinterpret_cast<int8_t *>(stage[0]);
-    int8_t *send_tile = reinterpret_cast<int8_t *>(stage[1]);
+    const SharedTile<Q> tile{reinterpret_cast<int8_t *>(stage[0]), reinterpret_cast<int8_t *>(stage[1])};
+    NoStats ns;
 
-    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        if (threadIdx.x == 0) queue_count = 0;
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
         __syncthreads();                                   // also: the previous tile has been flushed
-        const uint32_t first = tile * kThreads;
-        const uint32_t idx = first + threadIdx.x;
+        const uint32_t first = t * kThreads;
+        const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
         {
-            const bool active = idx < n_ranks;
-            const uint32_t a = rank_begin + (active ? idx : 0u);          // actual rank
-            const uint32_t r = a >= root ? a - root : a + (p - root);     // virtual rank
-            rows_or_enqueue<Q>(tab, g, r, active, ByteRow{recv_tile + threadIdx.x * Q},
-                               ByteRow{send_tile + threadIdx.x * Q}, threadIdx.x, want_recv, want_send,
-                               queue, &queue_count);
+            const bool active = threadIdx.x < rows;
+            const uint32_t a = rank_begin + first + (active ? threadIdx.x : 0u);   // actual rank
+            const uint32_t r = a >= root ? a - root : a + (p - root);              // virtual rank
+            rows_or_enqueue<Q>(tab, g, r, active, tile, threadIdx.x, rows, want_recv, want_send, queue, ns);
         }
         __syncthreads();
-        const int n_items = queue_count;
-        for (int i = threadIdx.x; i < n_items; i += kThreads) {
-            const SearchItem it = queue[i];
-            int8_t *tile_bytes = (it.dest & 1u) ? send_tile : recv_tile;
-            NoStats ns;
-            resolve_item(g, it, ByteRow{tile_bytes + (it.dest >> 1) * Q}, ns);
+        if (queue.n_search + queue.n_copy > 0) {           // the same for every thread
+            drain_queue(g, queue, tile, ns);
+            __syncthreads();
         }
-        if (n_items > 0) __syncthreads();                  // n_items is the same for every thread
-        const int rows = (int)min((uint32_t)kThreads, n_ranks - first);
         const size_t base = (size_t)first * (size_t)Q;
-        if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, rows * Q, recv_vec_ok, threadIdx.x);
-        if (want_send) flush_tile<kThreads>(stage[1], send_out + base, rows * Q, send_vec_ok, threadIdx.x);
+        if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, (int)rows * Q, recv_vec_ok, threadIdx.x);
+        if (want_send) flush_tile<kThreads>(stage[1], send_out + base, (int)rows * Q, send_vec_ok, threadIdx.x);
     }
 }
 
@@ -313,18 +376,27 @@ __device__ __forceinline__ void fill_tables(LevelTables &tab, const Geometry &g)
     }
 }
 
-// The sweep keeps the tables of one p round-major with p + 1 slots per round: slot p
-// takes the stand-in rows of lanes beyond the last rank.
+// The sweep's tile: kThreads consecutive ranks of the round-major tables of one p, which
+// have p + 1 slots per round; slot p takes the stand-in rows of lanes beyond the last rank.
+struct ScratchTile {
+    int8_t *recv_tab;
+    int8_t *send_tab;
+    uint32_t first;
+    uint32_t p;
+    __device__ __forceinline__ uint32_t slot(uint32_t i) const { return first + i < p ? first + i : p; }
+    __device__ __forceinline__ StridedColumn recv_row(uint32_t i) const
+    { return StridedColumn{recv_tab + slot(i), (size_t)p + 1u}; }
+    __device__ __forceinline__ StridedColumn send_row(uint32_t i) const
+    { return StridedColumn{send_tab + slot(i), (size_t)p + 1u}; }
+};
+
 template <int Q>
-__device__ __forceinline__ uint32_t sweep_rows(const LevelTables &tab, const Geometry &g, uint32_t r,
-                                               int8_t *recv_tab, int8_t *send_tab,
-                                               SearchItem *queue, int *queue_count)
+__device__ __forceinline__ uint32_t sweep_rows(const LevelTables &tab, const Geometry &g, const ScratchTile &tile,
+                                               uint32_t rows, TileQueue &queue, CountStats &stats)
 {
+    const uint32_t r = tile.first + threadIdx.x;
     const bool active = r < g.p;
-    const uint32_t slot = active ? r : g.p;
-    const size_t stride = (size_t)g.p + 1u;
-    return rows_or_enqueue<Q>(tab, g, active ? r : 1u, active, StridedColumn{recv_tab + slot, stride},
-                              StridedColumn{send_tab + slot, stride}, slot, true, true, queue, queue_count);
+    return rows_or_enqueue<Q>(tab, g, active ? r : 1u, active, tile, threadIdx.x, rows, true, true, queue, stats);
 }
 
 // Work queue: *queue_next counts values of p handed out, largest p first.
@@ -337,8 +409,7 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
     __shared__ uint64_t s_sum[kWarpsPerBlock];
     __shared__ uint32_t s_fail[8];
     __shared__ LevelTables s_tab;
-    __shared__ SearchItem queue[kThreads * kItemsPerRank];
-    __shared__ int queue_count;
+    __shared__ TileQueue queue;
     int8_t *tab = scratch + (size_t)blockIdx.x * scratch_per_block;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -366,35 +437,30 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
         int8_t *send_tab = tab + (size_t)q * stride;
         uint32_t fail[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
-        // the same closed-form pass and search queue as the table kernel, 256 ranks at a time
+        // the same closed-form pass and queues as the table kernel, 256 ranks at a time
         for (uint32_t first = 0; first < p; first += kThreads) {
-            if (threadIdx.x == 0) queue_count = 0;
+            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
             __syncthreads();
-            const uint32_t r = first + threadIdx.x;
-            {
-                uint32_t viol = 0;
-                switch (q) {
-#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, r, recv_tab, send_tab, queue, &queue_count); break;
-                    BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
-                    BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
-                    BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
-                    BCAST_CASE(19) BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24)
-                    BCAST_CASE(25) BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30)
-                    BCAST_CASE(31)
+            const ScratchTile tile{recv_tab, send_tab, first, p};
+            const uint32_t rows = min((uint32_t)kThreads, p - first);
+            CountStats st;
+            uint32_t viol = 0;
+            switch (q) {
+#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, tile, rows, queue, st); break;
+                BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
+                BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
+                BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
+                BCAST_CASE(19) BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24)
+                BCAST_CASE(25) BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30)
+                BCAST_CASE(31)
 #undef BCAST_CASE
-                }
-                if (__popc(viol) > 4) fail[4]++;
             }
+            if (__popc(viol) > 4) fail[4]++;
             __syncthreads();
-            const int n_items = queue_count;
-            for (int i = threadIdx.x; i < n_items; i += kThreads) {
-                const SearchItem it = queue[i];
-                int8_t *table = (it.dest & 1u) ? send_tab : recv_tab;
-                CountStats st;
-                resolve_item(g, it, StridedColumn{table + (it.dest >> 1), stride}, st);
-                if (st.s.descents > q - 1 || st.s.steps > 2 * q + st.s.descents) fail[5]++;
-                if (st.s.capped) fail[7]++;
-            }
+            drain_queue(g, queue, tile, st);
+            // Lemmas 5 and 6, summed over the searches this thread ran for the tile
+            if (st.s.capped) fail[7]++;
+            if (st.s.over_bound) fail[5]++;
         }
         __syncthreads();
 
@@ -496,7 +562,7 @@ static int64_t sweep_bytes_per_block(int32_t p_hi)
 
 constexpr int kSweepBlocksPerSm = 2;
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
-constexpr int kTableBlocksPerSm = 7;
+constexpr int kTableBlocksPerSm = 8;
 
 }  // namespace bcast
 

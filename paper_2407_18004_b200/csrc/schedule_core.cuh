@@ -62,22 +62,28 @@ __device__ __forceinline__ int baseblock(const Geometry &g, uint32_t r)
 
 // Counters the verification sweep reads; the table kernels pass a dummy.
 struct SearchStats {
-    int descents;       // recursive calls of Algorithm 4
-    int steps;          // list elements examined (Lemma 6 counts these)
-    int capped;         // the loop hit its safety cap
+    int descents;       // recursive calls of Algorithm 4 in the current search
+    int steps;          // list elements examined in the current search (Lemma 6 counts these)
+    int capped;         // some search hit the loop's safety cap
+    int over_bound;     // some search exceeded q-1 descents or 2q+R steps (Lemmas 5, 6)
 };
 
 struct NoStats {
+    __device__ __forceinline__ void begin() {}
     __device__ __forceinline__ void descent() {}
     __device__ __forceinline__ void step() {}
     __device__ __forceinline__ void cap() {}
+    __device__ __forceinline__ void end(int) {}
 };
 
 struct CountStats {
-    SearchStats s{0, 0, 0};
+    SearchStats s{0, 0, 0, 0};
+    __device__ __forceinline__ void begin() { s.descents = 0; s.steps = 0; }
     __device__ __forceinline__ void descent() { s.descents++; }
     __device__ __forceinline__ void step() { s.steps++; }
     __device__ __forceinline__ void cap() { s.capped = 1; }
+    __device__ __forceinline__ void end(int q)
+    { if (s.descents > q - 1 || s.steps > 2 * q + s.descents) s.over_bound = 1; }
 };
 
 // Algorithms 4 and 5 for virtual rank r with baseblock b.  emit(k, value) is
@@ -100,6 +106,7 @@ __device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b
     uint32_t sk_k1 = skip_of(g, 1);                       // skip[k+1]
     uint32_t m = 1u;                                      // max(skip[k], v+1)
     int guard = 6 * q + 16;                               // never reached; keeps the loop finite
+    stats.begin();
 
     while (true) {
         if (--guard < 0) { stats.cap(); return; }
@@ -123,7 +130,7 @@ __device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b
             accept = (u >= sk_k1);
             if (!accept) cand = 0u;                       // r' > R - skip[k+1]: return
         } else {
-            if (pending == 0u) return;                    // outermost call ran off the list
+            if (pending == 0u) { stats.end(q); return; }  // outermost call ran off the list
             bit = pending & (0u - pending);               // innermost pending call
             pending ^= bit;
             e = 31 - __clz(bit);
@@ -133,7 +140,7 @@ __device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b
         }
         if (accept) {
             emit(k, e == q ? b : e - q);
-            if (k == k_last) return;
+            if (k == k_last) { stats.end(q); return; }
             v = u - sk_e;                                 // s = r' + skip[e]
             remaining &= ~bit;
             cand = remaining & (bit - 1u);

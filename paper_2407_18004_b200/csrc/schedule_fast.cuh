@@ -48,10 +48,11 @@ template <> struct WalkInt<31> { typedef int64_t type; };
 // Rows of virtual rank r >= 1.  recv_row/send_row: (k, value) writers that can also
 // read back an entry.  Returns the rounds whose receive entry must come from the
 // search; *send_flags receives the rounds whose send entry must (Algorithm 6's
-// violations).
+// violations) and *baseblock_out the baseblock of r.
 template <int Q, class Row>
 __device__ __forceinline__ uint32_t closed_form_rows(const LevelTables &tab, uint32_t p, uint32_t r,
-                                                     Row recv_row, Row send_row, uint32_t *send_flags)
+                                                     Row recv_row, Row send_row, uint32_t *send_flags,
+                                                     int *baseblock_out)
 {
     typedef typename WalkInt<Q>::type Int;
     Int rp = (Int)r;                 // Algorithm 6: virtual processor index r'
@@ -114,6 +115,7 @@ __device__ __forceinline__ uint32_t closed_form_rows(const LevelTables &tab, uin
     recv_row(top, b);
     if (Q > 1 && top > 0 && recv_row.get(top - 1) == kMarkBase) recv_flags |= 1u << (top - 1);
     *send_flags = viol;
+    *baseblock_out = b;
     return recv_flags;
 }
 
