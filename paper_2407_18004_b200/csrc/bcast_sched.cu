@@ -28,6 +28,7 @@ namespace bcast {
 
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
+constexpr int kTableBlocksPerSm = 8;                   // resident blocks the table kernel is sized for
 constexpr int kMaxRowBytes = 32;                       // staged row: q <= 31 bytes (+ pad in batch form)
 
 // ------------------------------------------------------------------ per-rank rows
@@ -51,8 +52,7 @@ __device__ __forceinline__ int rank_rows(const Geometry &g, uint32_t r, Writer r
                                          bool want_recv, bool want_send, Stats &stats)
 {
     const int q = g.q;
-    const int b = baseblock(g, r);
-    if (want_recv) recv_search(g, r, b, q - 1, recv_row, stats);
+    const int b = want_recv ? recv_search_fast(g, r, q - 1, recv_row, stats) : baseblock(g, r);
     int nviol = 0;
     if (want_send) {
         if (r == 0u) {
@@ -112,8 +112,7 @@ __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t 
 // Work the closed-form pass leaves behind, collected per tile of kThreads consecutive ranks.
 //
 // SearchItem: recvblock[k] of virtual rank `rank` is wanted for every k in `mask` and goes
-// to row `row` of the tile's receive (table = 0) or send (table = 1) rows; base is the
-// rank's baseblock + 1 when the pass already knows it, else 0.
+// to row `row` of the tile's receive (table = 0) or send (table = 1) rows.
 // A copy (packed into 32 bits) says: sendblock[k] of row dst is recvblock[k] of row src of
 // the same tile (Section 2.3's definition, the to-processor being src), to be taken once
 // the searches of the tile are done.
@@ -121,8 +120,7 @@ struct SearchItem {
     uint32_t rank;
     uint32_t mask;
     uint16_t row;
-    uint8_t table;
-    uint8_t base;
+    uint16_t table;
 };
 
 constexpr int kSearchCapacity = 2 * kThreads;
@@ -139,10 +137,9 @@ struct TileQueue {
 template <class Row, class Stats>
 __device__ __forceinline__ void resolve_item(const Geometry &g, const SearchItem &it, Row row, Stats &stats)
 {
-    const int b = it.base != 0 ? (int)it.base - 1 : baseblock(g, it.rank);
     const uint32_t mask = it.mask;
-    recv_search(g, it.rank, b, 31 - __clz(mask),
-                [&](int k, int val) { if ((mask >> k) & 1u) row(k, val); }, stats);
+    recv_search_fast(g, it.rank, 31 - __clz(mask),
+                     [&](int k, int val) { if ((mask >> k) & 1u) row(k, val); }, stats);
 }
 
 // Queue a search; when the queue is full the calling thread does it on the spot.
@@ -185,7 +182,7 @@ __device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, cons
         b = Q;
     }
     if (want_recv && recv_flags != 0u)
-        push_search(g, queue, SearchItem{r, recv_flags, (uint16_t)index, 0, (uint8_t)(b + 1)}, tile, stats);
+        push_search(g, queue, SearchItem{r, recv_flags, (uint16_t)index, 0}, tile, stats);
     uint32_t todo = want_send ? send_flags : 0u;
     while (todo != 0u) {
         const int k = 31 - __clz(todo);
@@ -202,7 +199,7 @@ __device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, cons
         }
         uint32_t t = r + sk;
         if (t >= g.p) t -= g.p;
-        push_search(g, queue, SearchItem{t, 1u << k, (uint16_t)index, 1, 0}, tile, stats);
+        push_search(g, queue, SearchItem{t, 1u << k, (uint16_t)index, 1}, tile, stats);
     }
     return send_flags;
 }
@@ -239,7 +236,7 @@ struct SharedTile {
 };
 
 template <int Q>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
 schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t root,
                       uint32_t rank_begin, uint32_t n_ranks,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
@@ -562,7 +559,6 @@ static int64_t sweep_bytes_per_block(int32_t p_hi)
 
 constexpr int kSweepBlocksPerSm = 2;
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
-constexpr int kTableBlocksPerSm = 8;
 
 }  // namespace bcast
 

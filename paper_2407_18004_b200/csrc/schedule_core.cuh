@@ -86,27 +86,84 @@ struct CountStats {
     { if (s.descents > q - 1 || s.steps > 2 * q + s.descents) s.over_bound = 1; }
 };
 
-// Algorithms 4 and 5 for virtual rank r with baseblock b.  emit(k, value) is
-// called once for each k = 0..k_last in increasing order with the final schedule
-// value (b where the search accepted index q, else index - q).  k_last = q-1
-// yields the whole row; a smaller k_last stops early (used for one entry of
-// another rank's row).
+// State of the search of Algorithm 4 between two loop iterations.
+struct SearchState {
+    uint32_t remaining;   // list of skip indices still linked
+    uint32_t pending;     // indices of the calls in progress (the recursion stack)
+    uint32_t cand;        // part of the list the current call still has to scan
+    uint32_t u;           // R - r'
+    int b;                // baseblock of the rank
+};
+
+// Algorithm 5's set-up: all indices 0..q but the baseblock b, r' = 0, e = q.
+__device__ __forceinline__ SearchState search_from_top(const Geometry &g, uint32_t r, int b)
+{
+    SearchState s;
+    s.remaining = ((2u << g.q) - 1u) & ~(1u << b);
+    s.pending = 0u;
+    s.cand = s.remaining;
+    s.u = g.p + r;
+    s.b = b;
+    return s;
+}
+
+// The same search, entered where its first run of recursive calls ends.  While k = 0
+// the search descends on an index e exactly when skip[e] + 2 <= R - r', and R - r' is
+// then the part of R = p + r that the greedy decomposition of R over the skips
+// (skip[q] = p first) has not covered yet: every digit is descended on as long as at
+// least 2 remains after it, and every non-digit fails its test.  The walk below finds
+// that point with one compare per level instead of one search step, and the baseblock
+// on the way: the digit that leaves 0 is the baseblock (it is not in the list, the scan
+// goes on below it); a digit that leaves 1 is followed by digit 0 only, so the
+// baseblock is 0 and that digit is the next candidate.  The skipped steps and descents
+// are added to the counters so that the bounds of Lemmas 5 and 6 are still checked
+// against the whole search.
+template <class Stats>
+__device__ __forceinline__ SearchState search_from_digits(const Geometry &g, uint32_t r, Stats &stats)
+{
+    SearchState s;
+    uint32_t rem = g.p + r;
+    s.pending = 0u;
+    int k = g.q;
+    int b = 0;
+    for (;; --k) {
+        const uint32_t sk = skip_of(g, k);
+        if (rem >= sk) {
+            const uint32_t left = rem - sk;
+            if (left < 2u) { b = left == 0u ? k : 0; break; }
+            s.pending |= 1u << k;
+            rem = left;
+            stats.descent();
+        }
+        stats.step();
+    }
+    s.remaining = ((2u << g.q) - 1u) & ~(1u << b);
+    s.cand = s.remaining & ((2u << k) - 1u);
+    s.u = rem;
+    s.b = b;
+    return s;
+}
+
+// Algorithms 4 and 5 from a given state (k = 0, nothing accepted yet).  emit(k, value)
+// is called once for each k = 0..k_last in increasing order with the final schedule
+// value (b where the search accepted index q, else index - q).  k_last = q-1 yields
+// the whole row; a smaller k_last stops early.
 template <class Emit, class Stats>
-__device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b, int k_last,
-                                            Emit emit, Stats &stats)
+__device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchState &st, int k_last,
+                                                Emit emit, Stats &stats)
 {
     const int q = g.q;
-    uint32_t remaining = ((2u << q) - 1u) & ~(1u << b);   // list of skip indices, b unlinked
-    uint32_t pending = 0;                                 // indices of the calls in progress
-    uint32_t cand = remaining;                            // list part the current call still scans
-    uint32_t u = g.p + r;                                 // R - r'
+    const int b = st.b;
+    uint32_t remaining = st.remaining;
+    uint32_t pending = st.pending;
+    uint32_t cand = st.cand;
+    uint32_t u = st.u;                                    // R - r'
     uint32_t v = 0;                                       // R - s
     int k = 0;
     uint32_t sk_k = 1u;                                   // skip[k]
     uint32_t sk_k1 = skip_of(g, 1);                       // skip[k+1]
     uint32_t m = 1u;                                      // max(skip[k], v+1)
     int guard = 6 * q + 16;                               // never reached; keeps the loop finite
-    stats.begin();
 
     while (true) {
         if (--guard < 0) { stats.cap(); return; }
@@ -152,6 +209,26 @@ __device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b
     }
 }
 
+// Algorithms 4 and 5 for virtual rank r with baseblock b, as printed: from the top.
+template <class Emit, class Stats>
+__device__ __forceinline__ void recv_search(const Geometry &g, uint32_t r, int b, int k_last,
+                                            Emit emit, Stats &stats)
+{
+    stats.begin();
+    recv_search_run(g, search_from_top(g, r, b), k_last, emit, stats);
+}
+
+// The same result, entered after the first run of recursive calls.  Returns the baseblock.
+template <class Emit, class Stats>
+__device__ __forceinline__ int recv_search_fast(const Geometry &g, uint32_t r, int k_last,
+                                                Emit emit, Stats &stats)
+{
+    stats.begin();
+    const SearchState st = search_from_digits(g, r, stats);
+    recv_search_run(g, st, k_last, emit, stats);
+    return st.b;
+}
+
 // Algorithm 6 for virtual rank r > 0 with baseblock b: emit(k, value) for
 // k = q-1..1 and then k = 0.  Rounds the fast rules cannot decide are returned as
 // a bit set (at most four by Theorem 3); the caller fills those entries with
@@ -190,8 +267,7 @@ template <class Stats>
 __device__ __forceinline__ int recv_entry(const Geometry &g, uint32_t t, int k, Stats &stats)
 {
     int value = 0;
-    const int bt = baseblock(g, t);
-    recv_search(g, t, bt, k, [&](int kk, int val) { if (kk == k) value = val; }, stats);
+    recv_search_fast(g, t, k, [&](int kk, int val) { if (kk == k) value = val; }, stats);
     return value;
 }
 
