@@ -157,29 +157,91 @@ __device__ __forceinline__ void push_search(const Geometry &g, TileQueue &queue,
     }
 }
 
-// Rows of one rank through the closed forms; what the pass cannot decide is queued.
-// Called by every lane of a warp: lanes without a rank (`active` false) and the root
-// compute the rows of rank 1 as a stand-in, into their own row of the tile, and queue
-// nothing for them.  `index` is the rank's row in the tile, `rows` the tile's row count;
-// consecutive rows hold consecutive virtual ranks (mod p).  Returns Algorithm 6's violations.
-template <int Q, class Tile, class Stats>
-__device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, const Geometry &g, uint32_t r,
-                                                    bool active, const Tile &tile, uint32_t index, uint32_t rows,
-                                                    bool want_recv, bool want_send, TileQueue &queue, Stats &stats)
+// A send entry Algorithm 6 could not decide: round k of the rank in row `index`, virtual
+// rank r.  Its to-processor is a row of this tile whose receive entry will be final after
+// the tile's searches (then a copy is queued), or a rank that needs a search of its own.
+template <class Tile, class Stats>
+__device__ __forceinline__ void push_send_violation(const Geometry &g, uint32_t skip_k, int k, uint32_t r,
+                                                    uint32_t index, uint32_t rows, bool want_recv,
+                                                    TileQueue &queue, const Tile &tile, Stats &stats)
 {
-    const bool is_root = r == 0u;
-    uint32_t send_flags = 0;
-    int b = 0;
+    if (want_recv && index + skip_k < rows) {
+        const int slot = atomicAdd(&queue.n_copy, 1);
+        if (slot < kCopyCapacity) {
+            queue.copy[slot] = (index + skip_k) | (index << 9) | ((uint32_t)k << 18);
+            return;
+        }
+    }
+    uint32_t t = r + skip_k;
+    if (t >= g.p) t -= g.p;
+    push_search(g, queue, SearchItem{t, 1u << k, (uint16_t)index, 1}, tile, stats);
+}
+
+// Whether the ranks of a tile can share their high levels: a full tile of consecutive
+// virtual ranks without the root and without a wrap past p-1.
+template <int Q>
+__device__ __forceinline__ bool tile_can_share(const Geometry &g, uint32_t r_first, uint32_t rows)
+{
+    return Q >= kSharedFrom + 2 && rows == (uint32_t)kThreads && r_first >= 1u &&
+           r_first <= g.p - (uint32_t)kThreads;
+}
+
+// The closed-form pass for one tile: row i of the tile holds virtual rank (r_first + i) mod p,
+// `rows` rows are real.  Called by every thread of the block; thread i owns row i.  With a
+// run description of the tile (runs.n_runs > 0, see build_tile_runs) every rank copies its
+// high-level entries from it and walks only the low levels; without one each rank walks
+// all levels, with rank 1 as a stand-in for the root and for rows that are not real.  What
+// the pass cannot decide is queued.  Returns Algorithm 6's violations of this thread's rank.
+template <int Q, class Tile, class Stats>
+__device__ __forceinline__ uint32_t tile_pass(const LevelTables &tab, const Geometry &g,
+                                              const TileRuns<typename WalkInt<Q>::type> &runs,
+                                              uint32_t r_first, uint32_t rows, const Tile &tile,
+                                              bool want_recv, bool want_send, TileQueue &queue, Stats &stats)
+{
+    const uint32_t index = threadIdx.x;
+    const bool active = index < rows;
+    uint32_t r = 1u;
+    if (active) {
+        r = r_first + index;                               // < 2p: index < rows <= p
+        if (r >= g.p) r -= g.p;
+    }
     auto recv_row = tile.recv_row(index);
     auto send_row = tile.send_row(index);
-    uint32_t recv_flags = closed_form_rows<Q>(tab, g.p, (active && !is_root) ? r : 1u, recv_row, send_row,
-                                              &send_flags, &b);
-    if (!active) return 0u;
-    if (is_root) {                                          // the root sends block k in round k
-        for (int k = 0; k < Q; ++k) send_row(k, k);
-        recv_flags = (2u << (Q - 1)) - 1u;                  // and its receive row comes from the search
-        send_flags = 0u;
-        b = Q;
+    uint32_t recv_flags = 0, send_flags = 0;
+
+    bool shared = false;
+    if constexpr (Q >= kSharedFrom + 2) {
+        shared = runs.n_runs > 0;                          // the same for the whole block
+        if (shared) {
+            auto st = apply_tile_runs<Q>(runs, (int)index, recv_row, send_row);
+            closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
+            closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
+            // entries of the high levels that the description left undecided
+            if ((int)index < runs.n_pending) {
+                const uint32_t item = runs.pending[index];
+                const uint32_t row = item & 511u;
+                const int k = (int)((item >> 9) & 31u);
+                const uint32_t rr = r_first + row;
+                if ((item >> 14) & 1u) {
+                    stats.violation(row, k);
+                    if (want_send)
+                        push_send_violation(g, tab.skip[k], k, rr, row, rows, want_recv, queue, tile, stats);
+                } else if (want_recv) {
+                    push_search(g, queue, SearchItem{rr, 1u << k, (uint16_t)row, 0}, tile, stats);
+                }
+            }
+        }
+    }
+    if (!shared) {
+        const bool is_root = r == 0u;
+        int b = 0;
+        recv_flags = closed_form_rows<Q>(tab, g.p, is_root ? 1u : r, recv_row, send_row, &send_flags, &b);
+        if (!active) return 0u;
+        if (is_root) {                                     // the root sends block k in round k
+            for (int k = 0; k < Q; ++k) send_row(k, k);
+            recv_flags = (2u << (Q - 1)) - 1u;             // and its receive row comes from the search
+            send_flags = 0u;
+        }
     }
     if (want_recv && recv_flags != 0u)
         push_search(g, queue, SearchItem{r, recv_flags, (uint16_t)index, 0}, tile, stats);
@@ -187,19 +249,7 @@ __device__ __forceinline__ uint32_t rows_or_enqueue(const LevelTables &tab, cons
     while (todo != 0u) {
         const int k = 31 - __clz(todo);
         todo ^= 1u << k;
-        const uint32_t sk = tab.skip[k];
-        // the to-processor of round k: a row of this tile whose receive entry will be final
-        // after the tile's searches, or a rank that needs a search of its own
-        if (want_recv && index + sk < rows) {
-            const int slot = atomicAdd(&queue.n_copy, 1);
-            if (slot < kCopyCapacity) {
-                queue.copy[slot] = (index + sk) | (index << 9) | ((uint32_t)k << 18);
-                continue;
-            }
-        }
-        uint32_t t = r + sk;
-        if (t >= g.p) t -= g.p;
-        push_search(g, queue, SearchItem{t, 1u << k, (uint16_t)index, 1}, tile, stats);
+        push_send_violation(g, tab.skip[k], k, r, index, rows, want_recv, queue, tile, stats);
     }
     return send_flags;
 }
@@ -242,34 +292,62 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
                       int recv_vec_ok, int send_vec_ok)
 {
-    __shared__ uint32_t stage[2][kThreads * kMaxRowBytes / 4];
+    typedef typename WalkInt<Q>::type Int;
+    __shared__ uint32_t stage[2][(kThreads * Q + 15) / 16 * 4];   // byte tiles, kThreads rows of Q entries
     __shared__ TileQueue queue;
+    __shared__ LevelTables lookup;                         // the tables again, for per-lane indices
+    __shared__ TileRuns<Int> runs[kWarpsPerBlock];         // descriptions of the next kWarpsPerBlock tiles
     const Geometry g = make_geometry(p);
     const uint32_t n_tiles = (n_ranks + kThreads - 1u) / kThreads;
     const bool want_recv = recv_out != nullptr;
     const bool want_send = send_out != nullptr;
     const SharedTile<Q> tile{reinterpret_cast<int8_t *>(stage[0]), reinterpret_cast<int8_t *>(stage[1])};
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
     NoStats ns;
+    if (threadIdx.x <= Q) lookup.skip[threadIdx.x] = tab.skip[threadIdx.x];
+    if (threadIdx.x <= Q + 1) lookup.below[threadIdx.x] = tab.below[threadIdx.x];
+    __syncthreads();
 
-    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
-        __syncthreads();                                   // also: the previous tile has been flushed
-        const uint32_t first = t * kThreads;
-        const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
+    // tiles blockIdx.x, blockIdx.x + gridDim.x, ... in groups of kWarpsPerBlock: each warp first
+    // describes the runs of one tile of the group, then the block goes through the group
+    for (uint32_t group = blockIdx.x; group < n_tiles; group += gridDim.x * kWarpsPerBlock) {
         {
-            const bool active = threadIdx.x < rows;
-            const uint32_t a = rank_begin + first + (active ? threadIdx.x : 0u);   // actual rank
-            const uint32_t r = a >= root ? a - root : a + (p - root);              // virtual rank
-            rows_or_enqueue<Q>(tab, g, r, active, tile, threadIdx.x, rows, want_recv, want_send, queue, ns);
+            const uint32_t t = group + (uint32_t)warp * gridDim.x;
+            bool share = false;
+            if (t < n_tiles) {
+                const uint32_t first = t * kThreads;
+                const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
+                const uint32_t a = rank_begin + first;
+                const uint32_t r_first = a >= root ? a - root : a + (p - root);
+                share = tile_can_share<Q>(g, r_first, rows);
+                if constexpr (Q >= kSharedFrom + 2)
+                    if (share) build_tile_runs<Q>(tab, lookup, p, r_first, (int)rows, lane, runs[warp]);
+            }
+            if (!share && lane == 0) { runs[warp].n_runs = 0; runs[warp].n_pending = 0; }
         }
-        __syncthreads();
-        if (queue.n_search + queue.n_copy > 0) {           // the same for every thread
-            drain_queue(g, queue, tile, ns);
+        for (int slot = 0; slot < kWarpsPerBlock; ++slot) {
+            const uint32_t t = group + (uint32_t)slot * gridDim.x;
+            if (t >= n_tiles) break;
+            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
+            __syncthreads();                               // descriptions built; previous tile flushed
+            const uint32_t first = t * kThreads;
+            const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
+            {
+                const uint32_t a = rank_begin + first;                             // actual rank of row 0
+                const uint32_t r_first = a >= root ? a - root : a + (p - root);    // its virtual rank
+                tile_pass<Q>(tab, g, runs[slot], r_first, rows, tile, want_recv, want_send, queue, ns);
+            }
             __syncthreads();
+            if (queue.n_search + queue.n_copy > 0) {       // the same for every thread
+                drain_queue(g, queue, tile, ns);
+                __syncthreads();
+            }
+            const size_t base = (size_t)first * (size_t)Q;
+            if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, (int)rows * Q, recv_vec_ok, threadIdx.x);
+            if (want_send) flush_tile<kThreads>(stage[1], send_out + base, (int)rows * Q, send_vec_ok, threadIdx.x);
         }
-        const size_t base = (size_t)first * (size_t)Q;
-        if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, (int)rows * Q, recv_vec_ok, threadIdx.x);
-        if (want_send) flush_tile<kThreads>(stage[1], send_out + base, (int)rows * Q, send_vec_ok, threadIdx.x);
+        __syncthreads();                                   // the group's descriptions are free again
     }
 }
 
@@ -387,13 +465,52 @@ struct ScratchTile {
     { return StridedColumn{send_tab + slot(i), (size_t)p + 1u}; }
 };
 
+// Both tables of one p into the block's scratch, with the table kernel's own pass, queues
+// and run descriptions, kThreads ranks at a time.  Called by every thread of the block;
+// adds to the thread's failure counters [4] (violations), [5] (search bounds), [7] (cap).
 template <int Q>
-__device__ __forceinline__ uint32_t sweep_rows(const LevelTables &tab, const Geometry &g, const ScratchTile &tile,
-                                               uint32_t rows, TileQueue &queue, CountStats &stats)
+__device__ __forceinline__ void sweep_tables_of_p(const LevelTables &tab, const Geometry &g, int8_t *recv_tab,
+                                                  int8_t *send_tab, TileQueue &queue, void *runs_storage,
+                                                  uint32_t *row_viol, uint32_t *fail)
 {
-    const uint32_t r = tile.first + threadIdx.x;
-    const bool active = r < g.p;
-    return rows_or_enqueue<Q>(tab, g, active ? r : 1u, active, tile, threadIdx.x, rows, true, true, queue, stats);
+    typedef typename WalkInt<Q>::type Int;
+    TileRuns<Int> *runs = reinterpret_cast<TileRuns<Int> *>(runs_storage);
+    const uint32_t p = g.p;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    for (uint32_t group = 0; group < p; group += kThreads * kWarpsPerBlock) {
+        {
+            const uint32_t first = group + (uint32_t)warp * kThreads;
+            bool share = false;
+            if (first < p) {
+                const uint32_t rows = min((uint32_t)kThreads, p - first);
+                share = tile_can_share<Q>(g, first, rows);
+                if constexpr (Q >= kSharedFrom + 2)
+                    if (share) build_tile_runs<Q>(tab, tab, p, first, (int)rows, lane, runs[warp]);
+            }
+            if (!share && lane == 0) { runs[warp].n_runs = 0; runs[warp].n_pending = 0; }
+        }
+        for (int slot = 0; slot < kWarpsPerBlock; ++slot) {
+            const uint32_t first = group + (uint32_t)slot * kThreads;
+            if (first >= p) break;
+            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
+            row_viol[threadIdx.x] = 0u;
+            __syncthreads();
+            const ScratchTile tile{recv_tab, send_tab, first, p};
+            const uint32_t rows = min((uint32_t)kThreads, p - first);
+            CountStats st;
+            st.row_violations = row_viol;
+            uint32_t viol = tile_pass<Q>(tab, g, runs[slot], first, rows, tile, true, true, queue, st);
+            __syncthreads();
+            viol |= row_viol[threadIdx.x];                 // violations noted by the run descriptions
+            if (__popc(viol) > 4) fail[4]++;
+            drain_queue(g, queue, tile, st);
+            // Lemmas 5 and 6, over the searches this thread ran for the tile
+            if (st.s.capped) fail[7]++;
+            if (st.s.over_bound) fail[5]++;
+        }
+        __syncthreads();
+    }
 }
 
 // Work queue: *queue_next counts values of p handed out, largest p first.
@@ -406,6 +523,8 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
     __shared__ uint64_t s_sum[kWarpsPerBlock];
     __shared__ uint32_t s_fail[8];
     __shared__ LevelTables s_tab;
+    __shared__ uint32_t s_row_viol[kThreads];
+    __shared__ __align__(16) unsigned char s_runs[sizeof(TileRuns<int64_t>) * kWarpsPerBlock];
     __shared__ TileQueue queue;
     int8_t *tab = scratch + (size_t)blockIdx.x * scratch_per_block;
     const int lane = threadIdx.x & 31;
@@ -428,36 +547,22 @@ verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksu
         const Geometry g = make_geometry(p);
         const int q = g.q;
         fill_tables(s_tab, g);
+        __syncthreads();
         // tables of this p, round-major so that the checks read coalesced: tab[k*(p+1) + r]
         const size_t stride = (size_t)p + 1u;
         int8_t *recv_tab = tab;
         int8_t *send_tab = tab + (size_t)q * stride;
         uint32_t fail[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 
-        // the same closed-form pass and queues as the table kernel, 256 ranks at a time
-        for (uint32_t first = 0; first < p; first += kThreads) {
-            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
-            __syncthreads();
-            const ScratchTile tile{recv_tab, send_tab, first, p};
-            const uint32_t rows = min((uint32_t)kThreads, p - first);
-            CountStats st;
-            uint32_t viol = 0;
-            switch (q) {
-#define BCAST_CASE(N) case N: viol = sweep_rows<N>(s_tab, g, tile, rows, queue, st); break;
-                BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
-                BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
-                BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
-                BCAST_CASE(19) BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24)
-                BCAST_CASE(25) BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30)
-                BCAST_CASE(31)
+        switch (q) {
+#define BCAST_CASE(N) case N: sweep_tables_of_p<N>(s_tab, g, recv_tab, send_tab, queue, s_runs, s_row_viol, fail); break;
+            BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6)
+            BCAST_CASE(7) BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12)
+            BCAST_CASE(13) BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18)
+            BCAST_CASE(19) BCAST_CASE(20) BCAST_CASE(21) BCAST_CASE(22) BCAST_CASE(23) BCAST_CASE(24)
+            BCAST_CASE(25) BCAST_CASE(26) BCAST_CASE(27) BCAST_CASE(28) BCAST_CASE(29) BCAST_CASE(30)
+            BCAST_CASE(31)
 #undef BCAST_CASE
-            }
-            if (__popc(viol) > 4) fail[4]++;
-            __syncthreads();
-            drain_queue(g, queue, tile, st);
-            // Lemmas 5 and 6, summed over the searches this thread ran for the tile
-            if (st.s.capped) fail[7]++;
-            if (st.s.over_bound) fail[5]++;
         }
         __syncthreads();
 

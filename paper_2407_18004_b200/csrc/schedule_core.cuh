@@ -74,10 +74,14 @@ struct NoStats {
     __device__ __forceinline__ void step() {}
     __device__ __forceinline__ void cap() {}
     __device__ __forceinline__ void end(int) {}
+    __device__ __forceinline__ void violation(uint32_t, int) {}
 };
 
 struct CountStats {
     SearchStats s{0, 0, 0, 0};
+    uint32_t *row_violations = nullptr;     // per tile row: rounds another lane found undecided in Algorithm 6
+    __device__ __forceinline__ void violation(uint32_t row, int k)
+    { if (row_violations) atomicOr(row_violations + row, 1u << k); }
     __device__ __forceinline__ void begin() { s.descents = 0; s.steps = 0; }
     __device__ __forceinline__ void descent() { s.descents++; }
     __device__ __forceinline__ void step() { s.steps++; }
