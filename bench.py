@@ -134,19 +134,30 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle_sample(p: int, budget_ranks: int):
-    """The oracle as it stands on a window of ranks of the same p (single thread)."""
+def time_oracle_sample(p: int, budget_ranks: int, mode: str = "broadcast"):
+    """The oracle as it stands on a window of rows of the same workload (single thread)."""
     import oracle
     oracle.build()
     hi = min(budget_ranks, p)
     t0 = time.perf_counter()
-    oracle.schedule_table(p, 0, 0, hi)
+    if mode == "allbroadcast":
+        oracle.allbroadcast_schedule(p, p // 3, 0, hi)
+    else:
+        oracle.schedule_table(p, 0, 0, hi)
     dt = time.perf_counter() - t0
     full = (hi == p)
-    sample = ("all ranks of p=%d: receive rows by Algorithm 5, send rows gathered from them" % p) if full else (
-        "ranks [0,%d) of p=%d: receive row by Algorithm 5, send row by definition (q receive schedules per rank)"
-        % (hi, p))
+    what = "roots" if mode == "allbroadcast" else "ranks"
+    sample = ("all %s of p=%d: receive rows by Algorithm 5, send rows gathered from them" % (what, p)) if full else (
+        "%s [0,%d) of p=%d: receive row by Algorithm 5, send row by definition (q receive schedules per row)"
+        % (what, hi, p))
     return hi / dt, dt, sample
+
+
+def workload_label(mode: str, p: int, q: int) -> str:
+    if mode == "allbroadcast":
+        return ("Algorithm 7 tables of processor %d for all roots of p=%d (q=%d), recvblocks+sendblocks int32"
+                % (p // 3, p, q))
+    return "all ranks of p=%d (q=%d), root 0, recvblock+sendblock int32 tables" % (p, q)
 
 
 def oracle_sample_size(p: int) -> int:
@@ -165,22 +176,27 @@ def run_reference(args):
     per_step = min(per_step, p)
     import oracle
     oracle.build()
+    def ref_step():
+        if args.mode == "allbroadcast":
+            oracle.allbroadcast_schedule(p, p // 3, 0, per_step)
+        else:
+            oracle.schedule_table(p, 0, 0, per_step)
+
     for _ in range(args.warmup):
-        oracle.schedule_table(p, 0, 0, per_step)
+        ref_step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.schedule_table(p, 0, 0, per_step)
+        ref_step()
     dt = time.perf_counter() - t0
     value = per_step * args.steps / dt
-    sample = ("each step: ranks [0,%d) of p=%d, receive row by Algorithm 5, send row by definition"
-              % (per_step, p))
+    sample = ("each step: rows [0,%d) of the workload, receive row by Algorithm 5, send row by definition"
+              % per_step)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
         "data": "synthetic",
-        "config": {"workload": "all ranks of p=%d (q=%d), root 0, recvblock+sendblock int32 tables" % (p, q),
-                   "sampled": True},
+        "config": {"workload": workload_label(args.mode, p, q), "sampled": True},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -215,7 +231,10 @@ def run_ours(args):
 
     def step():
         bs.bcast_skips(p)
-        bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
+        if args.mode == "allbroadcast":
+            bs.bcast_allbroadcast_schedule(p, p // 3, 0, p, recv, send, stream)
+        else:
+            bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -255,7 +274,7 @@ def run_ours(args):
 
     # ---------------- end to end: host output tables through bcast_schedule_host
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.mode == "broadcast":
         staging = torch.empty(512 * 2 ** 20, dtype=torch.uint8, device="cuda")
         try:
             hrecv = torch.empty((p, q), dtype=torch.int32, pin_memory=True)
@@ -297,11 +316,11 @@ def run_ours(args):
     peak, peak_src = measured_peaks()
     kernel_ms = statistics.mean(per_step_ms)
     achieved = table_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = recorded_traffic("schedule_table_kernel", p)
+    traffic = recorded_traffic("schedule_table_kernel", p) if args.mode == "broadcast" else None
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        v, dt, sample = time_oracle_sample(p, oracle_sample_size(p))
+        v, dt, sample = time_oracle_sample(p, oracle_sample_size(p), args.mode)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                         "seconds": dt, "host_cores_available": os.cpu_count()}
 
@@ -309,7 +328,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": "all ranks of p=%d (q=%d), root 0, recvblock+sendblock int32 tables" % (p, q),
+        "config": {"workload": workload_label(args.mode, p, q),
                    "bytes_per_step": table_bytes, "replicas": world,
                    "l2": "tables larger than L2" if flush is None else "L2 flushed between steps"},
         "entries_per_s": value * 2 * q,
@@ -337,6 +356,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="p=2^27-1")
+    ap.add_argument("--mode", default="broadcast", choices=["broadcast", "allbroadcast"],
+                    help="broadcast: tables of all ranks for one root; allbroadcast: Algorithm 7's tables of one "
+                         "processor for all roots (no host-table leg)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

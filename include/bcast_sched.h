@@ -85,6 +85,20 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
                    int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);
 
 /*
+ * The schedule part of Algorithm 7 (all-broadcast, Appendix A) for one processor
+ * `rank`: with every processor j as root in turn, row j - root_begin of
+ * recvblocks_dev receives recvschedule((rank - j + p) mod p) and the same row of
+ * sendblocks_dev the send schedule for that root, which Algorithm 7 defines as
+ * sendblocks[j][k] = recvblocks[(j - skip[k] + p) mod p][k], for the roots j in
+ * [root_begin, root_end).  These are the rows of bcast_schedule's tables listed
+ * by descending virtual rank; layout, alignment, NULL rules, asynchrony and
+ * return value are those of bcast_schedule (BCAST_EINVAL_ROOT stands for a rank
+ * outside [0, p)).
+ */
+int bcast_allbroadcast_schedule(int32_t p, int32_t rank, int64_t root_begin, int64_t root_end,
+                                int32_t *recvblocks_dev, int32_t *sendblocks_dev, void *cuda_stream);
+
+/*
  * bcast_schedule with HOST output tables: the rank range is cut into chunks that
  * fit the caller's device staging buffer (staging_dev, staging_bytes, 16-byte
  * aligned; it must hold at least 32 rows of each requested table); each chunk

@@ -50,6 +50,7 @@ def _load():
             lib.oracle_sendschedule_def.argtypes = [i64, i64, i32p]
             lib.oracle_sendschedule_alg6.argtypes = [i64, i64, i32p, i32p, u64p]
             lib.oracle_schedule_table.argtypes = [i64, i64, i64, i64, i32p, i32p]
+            lib.oracle_allbroadcast_schedule.argtypes = [i64, i64, i64, i64, i32p, i32p]
             lib.oracle_round_k.argtypes = [ctypes.c_int, i64, i64]
             lib.oracle_round_block.argtypes = [ctypes.c_int, i64, i64, i32p]
             lib.oracle_round_block.restype = i64
@@ -139,6 +140,19 @@ def schedule_table(p: int, root: int = 0, rank_begin: int = 0, rank_end: int | N
                                        _i32(send) if want_send else None)
     if rc < 0:
         raise ValueError("bad arguments to schedule_table (%d)" % rc)
+    return recv, send
+
+
+def allbroadcast_schedule(p: int, r: int, root_begin: int = 0, root_end: int | None = None):
+    """Algorithm 7's (recvblocks, sendblocks) of processor r: row j-root_begin is for root j."""
+    if root_end is None:
+        root_end = p
+    q = q_of(p)
+    n = max(root_end - root_begin, 0)
+    recv = np.zeros((n, q), dtype=np.int32)
+    send = np.zeros((n, q), dtype=np.int32)
+    if _load().oracle_allbroadcast_schedule(p, r, root_begin, root_end, _i32(recv), _i32(send)) < 0:
+        raise ValueError("bad arguments to allbroadcast_schedule")
     return recv, send
 
 

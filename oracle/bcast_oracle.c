@@ -307,6 +307,44 @@ int oracle_schedule_table(int64_t p, int64_t root, int64_t rank_begin, int64_t r
 }
 
 /*
+ * Algorithm 7 (Appendix A), the schedule part, for processor r: with every
+ * processor j as root, recvblocks[j] = recvschedule((r - j + p) mod p), and then
+ * sendblocks[j][k] = recvblocks[(j - skip[k] + p) mod p][k].  Rows for the roots
+ * j in [root_begin, root_end); row-major, q entries per row.  When the whole
+ * range [0, p) is asked for the second loop reads this call's own recvblocks,
+ * as printed; for a window the needed rows of other roots are computed one
+ * receive schedule per entry.
+ */
+int oracle_allbroadcast_schedule(int64_t p, int64_t r, int64_t root_begin, int64_t root_end,
+                                 int32_t *recvblocks, int32_t *sendblocks)
+{
+    oracle_ctx c;
+    int tmp[ORACLE_MAXQ + 1], k, q;
+    int64_t j;
+    if (ctx_init_(&c, p)) return -1;
+    if (r < 0 || r >= p || root_begin < 0 || root_end > p || root_begin > root_end) return -1;
+    q = c.q;
+    if (q == 0) return 0;
+    for (j = root_begin; j < root_end; j++) {
+        int64_t rp = (r - j + p) % p;
+        recvschedule_(&c, rp, tmp, NULL);
+        for (k = 0; k < q; k++) recvblocks[(j - root_begin) * q + k] = tmp[k];
+    }
+    for (j = root_begin; j < root_end; j++) {
+        for (k = 0; k < q; k++) {
+            int64_t f = (j - c.skip[k] + p) % p;
+            if (root_begin == 0 && root_end == p) {
+                sendblocks[j * q + k] = recvblocks[f * q + k];
+            } else {
+                recvschedule_(&c, (r - f + p) % p, tmp, NULL);
+                sendblocks[(j - root_begin) * q + k] = tmp[k];
+            }
+        }
+    }
+    return q;
+}
+
+/*
  * Algorithm 1, the part that turns a schedule row into the block of one round.
  * n blocks, communication round j in [0, n-1+q): x = (q - (n-1) mod q) mod q
  * virtual rounds precede it, so i = x + j, k = i mod q, and after the shift by

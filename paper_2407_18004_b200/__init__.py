@@ -40,6 +40,7 @@ def _load():
         lib.bcast_skips.argtypes = [i32, vp]
         lib.bcast_schedule.argtypes = [i32, i32, i64, i64, vp, vp, vp]
         lib.bcast_schedule_host.argtypes = [i32, i32, i64, i64, vp, vp, vp, i64, vp]
+        lib.bcast_allbroadcast_schedule.argtypes = [i32, i32, i64, i64, vp, vp, vp]
         lib.bcast_schedule_batch.argtypes = [vp, vp, vp, i64, i32, vp, vp, vp, vp]
         lib.bcast_verify_sweep_scratch_bytes.argtypes = [i32, i32]
         lib.bcast_verify_sweep_scratch_bytes.restype = i64
@@ -117,6 +118,13 @@ def bcast_schedule(p: int, root: int, rank_begin: int, rank_end: int, recvblock,
                                          _stream(stream)))
 
 
+def bcast_allbroadcast_schedule(p: int, rank: int, root_begin: int, root_end: int, recvblocks, sendblocks,
+                                stream=None) -> int:
+    """Algorithm 7's tables of processor `rank`: row j-root_begin is its schedule with j as root. Returns q."""
+    return _check(_load().bcast_allbroadcast_schedule(p, rank, root_begin, root_end, _ptr(recvblocks),
+                                                      _ptr(sendblocks), _stream(stream)))
+
+
 def bcast_schedule_host(p: int, root: int, rank_begin: int, rank_end: int, recvblock_host, sendblock_host,
                         staging, stream=None) -> int:
     """Host (ideally pinned) int32 output tables, filled chunk by chunk through a device staging tensor."""
@@ -163,6 +171,19 @@ def schedule(p: int, root: int = 0, rank_begin: int = 0, rank_end: int | None = 
     recv = torch.empty((rows, q), dtype=torch.int32, device=device) if want_recv else None
     send = torch.empty((rows, q), dtype=torch.int32, device=device) if want_send else None
     bcast_schedule(p, root, rank_begin, rank_end, recv, send)
+    return recv, send
+
+
+def allbroadcast_schedule(p: int, rank: int, root_begin: int = 0, root_end: int | None = None, device="cuda"):
+    """Allocate and fill Algorithm 7's (recvblocks, sendblocks) of processor `rank` for the roots given."""
+    import torch
+    if root_end is None:
+        root_end = p
+    q = bcast_q(p)
+    rows = max(root_end - root_begin, 0)
+    recv = torch.empty((rows, q), dtype=torch.int32, device=device)
+    send = torch.empty((rows, q), dtype=torch.int32, device=device)
+    bcast_allbroadcast_schedule(p, rank, root_begin, root_end, recv, send)
     return recv, send
 
 

@@ -276,19 +276,25 @@ __device__ __forceinline__ void drain_queue(const Geometry &g, TileQueue &queue,
     }
 }
 
-// The table kernel's tile: byte rows in shared memory, laid out like the output.
+// The table kernel's tile: byte rows in shared memory, laid out like the output.  Row i of
+// the pass (ranks ascending) is output row i, or output row rows-1-i when the output lists
+// the ranks in descending order (the all-broadcast tables); rows beyond the real ones keep
+// their own slot.
 template <int Q>
 struct SharedTile {
     int8_t *recv;
     int8_t *send;
-    __device__ __forceinline__ ByteRow recv_row(uint32_t i) const { return ByteRow{recv + i * Q}; }
-    __device__ __forceinline__ ByteRow send_row(uint32_t i) const { return ByteRow{send + i * Q}; }
+    uint32_t rows;
+    bool descending;
+    __device__ __forceinline__ uint32_t slot(uint32_t i) const { return descending && i < rows ? rows - 1u - i : i; }
+    __device__ __forceinline__ ByteRow recv_row(uint32_t i) const { return ByteRow{recv + slot(i) * Q}; }
+    __device__ __forceinline__ ByteRow send_row(uint32_t i) const { return ByteRow{send + slot(i) * Q}; }
 };
 
 template <int Q>
 __global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
-schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t root,
-                      uint32_t rank_begin, uint32_t n_ranks,
+schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t anchor,
+                      uint32_t row_begin, uint32_t n_ranks, int descending,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
                       int recv_vec_ok, int send_vec_ok)
 {
@@ -301,7 +307,17 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
     const uint32_t n_tiles = (n_ranks + kThreads - 1u) / kThreads;
     const bool want_recv = recv_out != nullptr;
     const bool want_send = send_out != nullptr;
-    const SharedTile<Q> tile{reinterpret_cast<int8_t *>(stage[0]), reinterpret_cast<int8_t *>(stage[1])};
+    int8_t *const recv_bytes = reinterpret_cast<int8_t *>(stage[0]);
+    int8_t *const send_bytes = reinterpret_cast<int8_t *>(stage[1]);
+    // Output row x (global index row_begin + x) holds virtual rank (index - anchor) mod p, anchor
+    // being the root (bcast_schedule), or (anchor - index) mod p, anchor being the processor and
+    // the index the root (bcast_allbroadcast_schedule).  A tile's first virtual rank, ascending:
+    auto first_rank_of = [&](uint32_t first, uint32_t rows) {
+        const uint32_t lo = row_begin + first;
+        if (!descending) return lo >= anchor ? lo - anchor : lo + (p - anchor);
+        const uint32_t hi = lo + rows - 1u;
+        return anchor >= hi ? anchor - hi : anchor + (p - hi);
+    };
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     NoStats ns;
@@ -318,8 +334,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             if (t < n_tiles) {
                 const uint32_t first = t * kThreads;
                 const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
-                const uint32_t a = rank_begin + first;
-                const uint32_t r_first = a >= root ? a - root : a + (p - root);
+                const uint32_t r_first = first_rank_of(first, rows);
                 share = tile_can_share<Q>(g, r_first, rows);
                 if constexpr (Q >= kSharedFrom + 2)
                     if (share) build_tile_runs<Q>(tab, lookup, p, r_first, (int)rows, lane, runs[warp]);
@@ -333,11 +348,9 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             __syncthreads();                               // descriptions built; previous tile flushed
             const uint32_t first = t * kThreads;
             const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
-            {
-                const uint32_t a = rank_begin + first;                             // actual rank of row 0
-                const uint32_t r_first = a >= root ? a - root : a + (p - root);    // its virtual rank
-                tile_pass<Q>(tab, g, runs[slot], r_first, rows, tile, want_recv, want_send, queue, ns);
-            }
+            const SharedTile<Q> tile{recv_bytes, send_bytes, rows, descending != 0};
+            tile_pass<Q>(tab, g, runs[slot], first_rank_of(first, rows), rows, tile, want_recv, want_send,
+                         queue, ns);
             __syncthreads();
             if (queue.n_search + queue.n_copy > 0) {       // the same for every thread
                 drain_queue(g, queue, tile, ns);
@@ -710,30 +723,23 @@ int bcast_skips(int32_t p, int32_t *skip_host)
     return q;
 }
 
-int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
-                   int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream)
+// Launch of the table kernel for n_rows output rows starting at global row index row_begin.
+static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int64_t n_rows, int descending,
+                        int32_t *recv_dev, int32_t *send_dev, void *cuda_stream)
 {
-    if (p < 1) return BCAST_EINVAL_P;
-    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
-    if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
-    const int q = host_q(p);
-    const int64_t n_ranks = rank_end - rank_begin;
-    if (q == 0 || n_ranks == 0) return q;              // zero-size tables: nothing to write
-    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
-    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
     const int sms = sm_count();
     if (sms <= 0) return BCAST_ECUDA;
-    const int64_t n_tiles = (n_ranks + kThreads - 1) / kThreads;
+    const int64_t n_tiles = (n_rows + kThreads - 1) / kThreads;
     const int64_t grid_cap = (int64_t)sms * kTableBlocksPerSm;
     const int grid = (int)(n_tiles < grid_cap ? n_tiles : grid_cap);
     const LevelTables tab = host_tables(p, q);
-    const int recv_vec = ((uintptr_t)recvblock_dev & 15u) == 0, send_vec = ((uintptr_t)sendblock_dev & 15u) == 0;
+    const int recv_vec = ((uintptr_t)recv_dev & 15u) == 0, send_vec = ((uintptr_t)send_dev & 15u) == 0;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     switch (q) {
 #define BCAST_CASE(N)                                                                                     \
     case N:                                                                                               \
-        schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)root,         \
-            (uint32_t)rank_begin, (uint32_t)n_ranks, recvblock_dev, sendblock_dev, recv_vec, send_vec);   \
+        schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)anchor,       \
+            (uint32_t)row_begin, (uint32_t)n_rows, descending, recv_dev, send_dev, recv_vec, send_vec);   \
         break;
         BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6) BCAST_CASE(7)
         BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12) BCAST_CASE(13)
@@ -745,6 +751,34 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
     }
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
+}
+
+int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
+                   int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
+    if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
+    const int q = host_q(p);
+    const int64_t n_ranks = rank_end - rank_begin;
+    if (q == 0 || n_ranks == 0) return q;              // zero-size tables: nothing to write
+    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
+    return launch_table(p, q, root, rank_begin, n_ranks, 0, recvblock_dev, sendblock_dev, cuda_stream);
+}
+
+int bcast_allbroadcast_schedule(int32_t p, int32_t rank, int64_t root_begin, int64_t root_end,
+                                int32_t *recvblocks_dev, int32_t *sendblocks_dev, void *cuda_stream)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (rank < 0 || rank >= p) return BCAST_EINVAL_ROOT;
+    if (root_begin < 0 || root_begin > root_end || root_end > p) return BCAST_EINVAL_RANGE;
+    const int q = host_q(p);
+    const int64_t n_roots = root_end - root_begin;
+    if (q == 0 || n_roots == 0) return q;
+    if (recvblocks_dev == nullptr && sendblocks_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)recvblocks_dev & 3u) || ((uintptr_t)sendblocks_dev & 3u)) return BCAST_EALIGN;
+    return launch_table(p, q, rank, root_begin, n_roots, 1, recvblocks_dev, sendblocks_dev, cuda_stream);
 }
 
 int bcast_schedule_host(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,

@@ -272,3 +272,36 @@ def test_schedule_host_chunks():
     assert_equal("host send part", part.numpy(), osend[777:5777])
     with pytest.raises(bs.BcastError):
         bs.bcast_schedule_host(p, root, 0, p, recv, send, staging[:1024])
+
+
+# ------------------------------------------------------------------ Algorithm 7: all-broadcast tables
+@pytest.mark.parametrize("p,rank", [(2, 1), (17, 5), (1000, 0), (1000, 999), (1000, 417), (5000, 1234),
+                                    (70001, 69999), (2 ** 16 + 1, 3)])
+def test_allbroadcast_tables(p, rank):
+    orecv, osend = oracle.allbroadcast_schedule(p, rank)
+    recv, send = bs.allbroadcast_schedule(p, rank)
+    torch.cuda.synchronize()
+    assert_equal("recvblocks", recv.cpu().numpy(), orecv)
+    assert_equal("sendblocks", send.cpu().numpy(), osend)
+    for lo, hi in [(0, 1), (p - 1, p), (p // 3, min(p, p // 3 + 300)), (1, 1)]:
+        recv, send = bs.allbroadcast_schedule(p, rank, lo, hi)
+        torch.cuda.synchronize()
+        assert_equal(f"recvblocks[{lo}:{hi}]", recv.cpu().numpy(), orecv[lo:hi])
+        assert_equal(f"sendblocks[{lo}:{hi}]", send.cpu().numpy(), osend[lo:hi])
+
+
+def test_allbroadcast_large_p_is_the_reversed_broadcast_table():
+    """p = 2^20+1: row j of processor r's tables is row (r - j) mod p of the root-0 tables."""
+    p, rank = workloads.P_MEDIUM, 777777
+    recv0, send0 = bs.schedule(p)
+    recv, send = bs.allbroadcast_schedule(p, rank)
+    torch.cuda.synchronize()
+    idx = (rank - torch.arange(p, device="cuda")) % p
+    assert bool((recv == recv0[idx]).all()) and bool((send == send0[idx]).all())
+    # and a window against the oracle, entry by entry
+    lo, hi = 500000, 501000
+    orecv, osend = oracle.allbroadcast_schedule(p, rank, lo, hi)
+    assert_equal("recvblocks", recv[lo:hi].cpu().numpy(), orecv)
+    assert_equal("sendblocks", send[lo:hi].cpu().numpy(), osend)
+    with pytest.raises(bs.BcastError):
+        bs.allbroadcast_schedule(p, p)

@@ -392,3 +392,70 @@ def test_batch_form():
         assert recv[i, :q].tolist() == oracle.recvschedule(int(p[i]), r).tolist()
         assert send[i, :q].tolist() == oracle.sendschedule_alg6(int(p[i]), r)[0].tolist()
         assert (recv[i, q:] == oracle.PAD).all() and (send[i, q:] == oracle.PAD).all()
+
+
+# ---------------------------------------------------------------- Algorithm 7: all-broadcast tables
+def test_allbroadcast_tables_are_renumbered_broadcast_tables():
+    """Processor r with root j is virtual rank (r - j) mod p of the broadcast from root j."""
+    for p in [2, 3, 9, 17, 18, 100, 257]:
+        per_root = [oracle.schedule_table(p, root) for root in range(p)]
+        for r in sorted({0, 1, p // 2, p - 1}):
+            recv, send = oracle.allbroadcast_schedule(p, r)
+            for j in range(p):
+                assert recv[j].tolist() == per_root[j][0][r].tolist()
+                assert send[j].tolist() == per_root[j][1][r].tolist()
+            lo, hi = p // 3, min(p, p // 3 + 7)
+            recv_w, send_w = oracle.allbroadcast_schedule(p, r, lo, hi)
+            assert np.array_equal(recv_w, recv[lo:hi]) and np.array_equal(send_w, send[lo:hi])
+
+
+def test_allbroadcast_simulation():
+    """Algorithm 7 round by round on tiny systems: every processor ends with all n blocks of every
+    other processor after n-1+q rounds, what it unpacks for root j is what its from-processor packed
+    for root j, and nobody packs a block it does not hold."""
+    for p in list(range(2, 14)) + [17, 18]:
+        q = oracle.q_of(p)
+        skip = oracle.skips(p)
+        tables = [oracle.allbroadcast_schedule(p, r) for r in range(p)]
+        for n in (1, 2, 3, 5, 8):
+            x = (q - (n - 1) % q) % q
+            held = np.zeros((p, p, n), dtype=bool)          # held[r][j][b]: r has block b of root j
+            for r in range(p):
+                held[r, r, :] = True
+            # Algorithm 7's shift of all entries by -x, +q for the rounds before x
+            sched = []
+            for r in range(p):
+                recv = tables[r][0].astype(np.int64) - x
+                send = tables[r][1].astype(np.int64) - x
+                recv[:, :x] += q
+                send[:, :x] += q
+                sched.append((recv, send))
+            for i in range(x, n + q - 1 + x):
+                k = i % q
+                packed = {}
+                for r in range(p):
+                    t = (r + int(skip[k])) % p
+                    for j in range(p):
+                        if j != t:
+                            raw = int(sched[r][1][j, k])
+                            if raw >= 0:
+                                blk = min(raw, n - 1)
+                                assert held[r, j, blk], (p, n, i, r, j, blk)
+                                packed[(r, j)] = blk
+                        sched[r][1][j, k] += q
+                arrivals = []
+                for r in range(p):
+                    f = (r - int(skip[k])) % p
+                    for j in range(p):
+                        if j != r:
+                            raw = int(sched[r][0][j, k])
+                            if raw >= 0:
+                                blk = min(raw, n - 1)
+                                assert packed.get((f, j)) == blk, (p, n, i, r, j, blk, packed.get((f, j)))
+                                arrivals.append((r, j, blk))
+                            else:
+                                assert (f, j) not in packed or j == r, (p, n, i, r, j)
+                        sched[r][0][j, k] += q
+                for r, j, blk in arrivals:
+                    held[r, j, blk] = True
+            assert held.all(), (p, n)
