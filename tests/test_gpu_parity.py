@@ -305,3 +305,30 @@ def test_allbroadcast_large_p_is_the_reversed_broadcast_table():
     assert_equal("sendblocks", send[lo:hi].cpu().numpy(), osend)
     with pytest.raises(bs.BcastError):
         bs.allbroadcast_schedule(p, p)
+
+
+# ------------------------------------------------------------------ largest sizes: q = 30 and 31 (64-bit walk)
+@pytest.mark.parametrize("p", [2 ** 31 - 1, 2 ** 30 + 1, 2 ** 30, 2 ** 31 - 5, 1431655765])
+def test_rank_windows_of_the_largest_p(p):
+    """Windows of ranks of p near 2^31, where p + r passes 2^31: both ends, around skips, a wrap past
+    the root, and random places; every window spans several tiles and ends ragged."""
+    q = bs.bcast_q(p)
+    skips = bs.bcast_skips(p)
+    rng = np.random.default_rng(p % 1000)
+    root = int(rng.integers(0, p))
+    starts = [0, p - 1500, root - 700 if root >= 700 else 0, int(skips[q - 1]) - 600, int(skips[q - 2]) + root - 300]
+    starts += [int(x) for x in rng.integers(0, p - 2000, 3)]
+    for lo in starts:
+        lo = max(0, min(lo, p - 1500))
+        hi = lo + 1500 - (lo % 7)
+        recv, send = bs.schedule(p, root, lo, hi)
+        torch.cuda.synchronize()
+        orecv, osend = oracle.schedule_table(p, root, lo, hi)
+        assert_equal(f"p={p} recv[{lo}:{hi}]", recv.cpu().numpy(), orecv)
+        assert_equal(f"p={p} send[{lo}:{hi}]", send.cpu().numpy(), osend)
+    lo = p - 3000
+    arecv, asend = bs.allbroadcast_schedule(p, root, lo, p)
+    torch.cuda.synchronize()
+    oarecv, oasend = oracle.allbroadcast_schedule(p, root, lo, p)
+    assert_equal("allbroadcast recv", arecv.cpu().numpy(), oarecv)
+    assert_equal("allbroadcast send", asend.cpu().numpy(), oasend)
