@@ -38,7 +38,9 @@ def _load():
     global _lib
     with _lock:
         if _lib is None:
-            lib = ctypes.CDLL(build())
+            # ORACLE_LIBRARY: a deliberately broken build, used only by the test that checks that the
+            # pins notice planted mistakes
+            lib = ctypes.CDLL(os.environ.get("ORACLE_LIBRARY") or build())
             i32p = ctypes.POINTER(ctypes.c_int32)
             i64p = ctypes.POINTER(ctypes.c_int64)
             u64p = ctypes.POINTER(ctypes.c_uint64)
