@@ -130,7 +130,9 @@ __device__ __forceinline__ SearchState search_from_digits(const Geometry &g, uin
     s.pending = 0u;
     int k = g.q;
     int b = 0;
-    for (;; --k) {
+    // ends at level 1 at the latest (the remainder entering level k is below skip[k+1], so it is 2
+    // or 3 there); the bound on k only keeps the loop finite whatever happens
+    for (; k > 0; --k) {
         const uint32_t sk = skip_of(g, k);
         if (rem >= sk) {
             const uint32_t left = rem - sk;
