@@ -840,7 +840,9 @@ int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const in
     if (sms <= 0) return BCAST_ECUDA;
     const int64_t n_tiles = (nq + 31) / 32;
     const int64_t blocks_needed = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const int64_t grid_cap = (int64_t)sms * kTableBlocksPerSm;
+    // one warp tile per warp while that keeps the grid below 2^20 blocks: short-lived blocks
+    // balance better than a resident grid striding over the tiles
+    const int64_t grid_cap = (int64_t)1 << 20;
     const int grid = (int)(blocks_needed < grid_cap ? blocks_needed : grid_cap);
     schedule_batch_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
         p_dev, rank_dev, root_dev, nq, row_stride, recvblock_dev, sendblock_dev, bad_count_dev,
