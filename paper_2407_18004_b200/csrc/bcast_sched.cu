@@ -29,6 +29,7 @@ namespace bcast {
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kTableBlocksPerSm = 8;                   // resident blocks the table kernel is sized for
+constexpr int kSweepBlocksPerSm = 4;                   // resident blocks of the verification sweep
 constexpr int kBlocksPerSmWanted = 64;                 // grid size below which blocks take fewer tiles
 constexpr int kMaxRowBytes = 32;                       // staged row: q <= 31 bytes (+ pad in batch form)
 
@@ -528,7 +529,7 @@ __device__ __forceinline__ void sweep_tables_of_p(const LevelTables &tab, const 
 }
 
 // Work queue: *queue_next counts values of p handed out, largest p first.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kSweepBlocksPerSm)
 verify_sweep_kernel(uint32_t p_lo, uint32_t p_hi, uint64_t *__restrict__ checksum_out,
                     uint32_t *__restrict__ fail_counts, int8_t *scratch,
                     size_t scratch_per_block, unsigned int *queue_next)
@@ -676,7 +677,6 @@ static int64_t sweep_bytes_per_block(int32_t p_hi)
     return round_up((int64_t)2 * host_q(p_hi) * ((int64_t)p_hi + 1), 256);
 }
 
-constexpr int kSweepBlocksPerSm = 2;
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
 
 }  // namespace bcast
