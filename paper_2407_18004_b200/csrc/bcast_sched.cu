@@ -1,20 +1,25 @@
 // C ABI and kernels of the broadcast-schedule library (see include/bcast_sched.h).
 //
 // Kernels
-//   schedule_table_kernel   one thread per rank, one warp per tile of 32 consecutive
-//                           ranks.  Each lane computes its receive row (Algorithms
-//                           3-5) and send row (Algorithm 6) in registers and drops the
-//                           entries as bytes into a per-warp shared-memory tile laid
-//                           out exactly like the output (row-major, q entries per row).
-//                           The warp then widens the tile to int32 and streams it out
-//                           as one contiguous run of 16-byte stores, so every store
-//                           instruction fills whole 32-byte sectors.  No block-wide
-//                           barrier: warps never wait for each other.
-//   schedule_batch_kernel   the same per-thread computation for independent
-//                           (p, rank, root) queries, rows padded to row_stride.
-//   verify_sweep_kernel     persistent blocks pull values of p from a queue, build the
-//                           tables of one p in scratch memory, then check the paper's
-//                           correctness conditions against them and reduce a checksum.
+//   schedule_table_kernel   one thread per rank, one block per run of up to 8 tiles of 256
+//                           consecutive ranks.  The ranks of a tile agree on their digits at
+//                           the high levels over long runs, so one warp describes those runs
+//                           once (a lane per level) and every thread copies its rank's
+//                           high-level entries from the description and walks only the low
+//                           levels with the closed forms (schedule_fast.cuh).  Entries land as
+//                           bytes in a shared-memory tile laid out exactly like the output;
+//                           what the closed forms leave undecided is collected in shared-
+//                           memory queues and resolved by the search of Algorithms 4 and 5
+//                           (schedule_core.cuh) or copied from a neighbouring row.  The block
+//                           then widens the tile to int32 and streams it out as one
+//                           contiguous run of 16-byte stores, so every store instruction
+//                           fills whole 32-byte sectors.
+//   schedule_batch_kernel   independent (p, rank, root) queries, one per thread: receive row by
+//                           the search, send row by Algorithm 6; rows padded to row_stride.
+//   verify_sweep_kernel     persistent blocks pull values of p from a queue, build the tables
+//                           of one p in scratch memory with the table kernel's device
+//                           functions, then check the paper's correctness conditions against
+//                           them and reduce a checksum.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
