@@ -332,3 +332,26 @@ def test_rank_windows_of_the_largest_p(p):
     oarecv, oasend = oracle.allbroadcast_schedule(p, root, lo, p)
     assert_equal("allbroadcast recv", arecv.cpu().numpy(), oarecv)
     assert_equal("allbroadcast send", asend.cpu().numpy(), oasend)
+
+
+# ------------------------------------------------------------------ tiles that cannot share their high levels
+@pytest.mark.parametrize("p", [100003, 2 ** 17 + 1, 2 ** 17 - 1])
+def test_windows_roots_and_single_tables_mid_p(p):
+    """q = 17, 18: full tiles take the shared run descriptions; the windows below also produce tiles
+    that hold the root, wrap past p-1, start off a multiple of 256 and end ragged, and launches that
+    want only one of the two tables (no in-tile copies of receive entries then)."""
+    q = bs.bcast_q(p)
+    for root in (0, 1, 255, 256, 50000, p - 1):
+        orecv, osend = oracle.schedule_table(p, root)
+        for lo, hi in [(0, p), (1, 4099), (root, min(p, root + 777)), (max(0, root - 300), min(p, root + 300)),
+                       (p - 1000, p), (12345, 12345 + 2048)]:
+            recv, send = bs.schedule(p, root, lo, hi)
+            torch.cuda.synchronize()
+            assert_equal(f"root {root} recv[{lo}:{hi}]", recv.cpu().numpy(), orecv[lo:hi])
+            assert_equal(f"root {root} send[{lo}:{hi}]", send.cpu().numpy(), osend[lo:hi])
+        recv, _ = bs.schedule(p, root, 3, p - 5, want_send=False)
+        _, send = bs.schedule(p, root, 3, p - 5, want_recv=False)
+        torch.cuda.synchronize()
+        assert_equal("recv only", recv.cpu().numpy(), orecv[3:p - 5])
+        assert_equal("send only", send.cpu().numpy(), osend[3:p - 5])
+        assert recv.shape == (p - 8, q)
