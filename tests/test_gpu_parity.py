@@ -355,3 +355,26 @@ def test_windows_roots_and_single_tables_mid_p(p):
         assert_equal("recv only", recv.cpu().numpy(), orecv[3:p - 5])
         assert_equal("send only", send.cpu().numpy(), osend[3:p - 5])
         assert recv.shape == (p - 8, q)
+
+
+# ------------------------------------------------------------------ two device implementations against each other
+@pytest.mark.parametrize("p,root", [(2 ** 24 + 3, 0), (2 ** 24 + 3, 9999999), (123456789, 1), (2 ** 27 - 1, 5)])
+def test_table_kernel_against_batch_kernel_at_scale(p, root):
+    """Every entry of 2^24 consecutive ranks: the table kernel (closed forms, shared high levels, queues)
+    against the batch kernel (search of Algorithms 4/5 and Algorithm 6 per thread).  Both are compared
+    with the oracle elsewhere; here they must agree with each other where the oracle is too slow."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * 2 ** 30:
+        pytest.skip("needs 12 GB of device memory")
+    n = min(p, 2 ** 24)
+    q = bs.bcast_q(p)
+    lo = (p - n) // 2
+    recv, send = bs.schedule(p, root, lo, lo + n)
+    ranks = torch.arange(lo, lo + n, dtype=torch.int32, device="cuda")
+    ps = torch.full((n,), p, dtype=torch.int32, device="cuda")
+    roots = torch.full((n,), root, dtype=torch.int32, device="cuda")
+    brecv, bsend, bad = bs.schedule_batch(ps, ranks, roots, 31)
+    torch.cuda.synchronize()
+    assert int(bad) == 0
+    assert bool((recv == brecv[:, :q]).all()), "receive tables differ"
+    assert bool((send == bsend[:, :q]).all()), "send tables differ"
