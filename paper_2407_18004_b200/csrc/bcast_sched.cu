@@ -157,10 +157,8 @@ __device__ __forceinline__ void push_search(const Geometry &g, TileQueue &queue,
     const int slot = atomicAdd(&queue.n_search, 1);
     if (slot < kSearchCapacity) {
         queue.search[slot] = it;
-    } else if (it.table == 0) {
-        resolve_item(g, it, tile.recv_row(it.row), stats);
     } else {
-        resolve_item(g, it, tile.send_row(it.row), stats);
+        resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
     }
 }
 
@@ -270,8 +268,8 @@ __device__ __forceinline__ void drain_queue(const Geometry &g, TileQueue &queue,
     const int n_copy = min(queue.n_copy, kCopyCapacity);
     for (int i = threadIdx.x; i < n_search; i += kThreads) {
         const SearchItem it = queue.search[i];
-        if (it.table == 0) resolve_item(g, it, tile.recv_row(it.row), stats);
-        else resolve_item(g, it, tile.send_row(it.row), stats);
+        // one call site: items for either table run the same instructions side by side
+        resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
     }
     if (n_copy > 0) {
         __syncthreads();                                   // n_copy is the same for every thread
