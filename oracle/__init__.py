@@ -49,6 +49,7 @@ def _load():
             lib.oracle_skips.argtypes = [i64, i64p]
             lib.oracle_baseblock.argtypes = [i64, i64]
             lib.oracle_recvschedule.argtypes = [i64, i64, i32p, i64p]
+            lib.oracle_recv_positions.argtypes = [i64, i64, i64p]
             lib.oracle_sendschedule_def.argtypes = [i64, i64, i32p]
             lib.oracle_sendschedule_alg6.argtypes = [i64, i64, i32p, i32p, u64p]
             lib.oracle_schedule_table.argtypes = [i64, i64, i64, i64, i32p, i32p]
@@ -106,6 +107,15 @@ def recvschedule(p: int, r: int, with_stats: bool = False):
         return out, dict(calls=int(st[0]), iters=int(st[1]), retests=int(st[2]),
                          retest_hits=int(st[3]), oob=int(st[4]))
     return out
+
+
+def recv_positions(p: int, r: int) -> np.ndarray:
+    """The processors r'_k of Lemma 4 (numbered in [p, 2p)) behind each receive entry of r."""
+    q = q_of(p)
+    out = np.zeros(max(q, 1), dtype=np.int64)
+    if _load().oracle_recv_positions(p, r, _i64(out)) < 0:
+        raise ValueError("bad (p, r)")
+    return out[:q]
 
 
 def sendschedule(p: int, r: int) -> np.ndarray:

@@ -56,6 +56,7 @@ typedef struct {
                             very index its caller just tested                 */
     int64_t  retest_hits;/* how many of those passed the outer test           */
     int64_t  oob;        /* skip[k+1] wanted with k >= q                      */
+    int64_t  rprime[ORACLE_MAXQ + 1];  /* the processor r'_k accepted for round k (Lemma 4) */
 } oracle_ctx;
 
 #define NEXT(c, e) ((c)->next_[(e) + 1])
@@ -118,6 +119,7 @@ static int allblocks_(oracle_ctx *c, int64_t r, int64_t rp, int64_t s, int e, in
             if (k >= c->q) { c->oob++; return k; }
             if (rp > r - skip[k + 1]) return k;
             s = rp + skip[e];
+            c->rprime[k] = s;
             c->recvblock[k] = e;
             k = k + 1;
             NEXT(c, PREV(c, e)) = NEXT(c, e);
@@ -180,6 +182,21 @@ int oracle_recvschedule(int64_t p, int64_t r, int32_t *recvblock, int64_t *stats
         stats[0] = c.calls; stats[1] = c.iters; stats[2] = c.retests;
         stats[3] = c.retest_hits; stats[4] = c.oob;
     }
+    return c.q;
+}
+
+/*
+ * The intermediate processors r'_k (in [p, 2p), the search runs on p + r) whose
+ * baseblocks make up the receive schedule of r: Lemma 4 places them in
+ * [p + r - skip[k+1], p + r - skip[k]].
+ */
+int oracle_recv_positions(int64_t p, int64_t r, int64_t *rprime)
+{
+    oracle_ctx c;
+    int tmp[ORACLE_MAXQ + 1], k;
+    if (ctx_init_(&c, p) || r < 0 || r >= p) return -1;
+    recvschedule_(&c, r, tmp, NULL);
+    for (k = 0; k < c.q; k++) rprime[k] = c.rprime[k];
     return c.q;
 }
 

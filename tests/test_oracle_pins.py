@@ -271,6 +271,29 @@ def test_search_bounds():
             assert (row > -1000 + 64).all()                         # every entry was written
 
 
+def test_lemma4_intermediate_processors():
+    """Lemma 4: r - skip[k+1] <= r'_k <= r - skip[k] (on p + r), strictly decreasing in k, and
+    recvblock[k] is the baseblock of r'_k (the root's own index q standing for b)."""
+    ps = list(range(2, 300)) + BIG_P
+    for p in ps:
+        s = oracle.skips(p).tolist()
+        q = len(s) - 1
+        ranks = range(p) if p < 300 else [0, 1, p - 1] + [int(x) for x in RNG.integers(0, p, 100)]
+        for r in ranks:
+            pos = oracle.recv_positions(p, r).tolist()
+            row = oracle.recvschedule(p, r).tolist()
+            b = oracle.baseblock(p, r)
+            for k in range(q):
+                assert p + r - s[k + 1] <= pos[k] <= p + r - s[k], (p, r, k)
+                if k > 0:
+                    assert pos[k] < pos[k - 1]
+                # the accepted index is the first index of the path to r'_k, which starts with skip[q] = p
+                if pos[k] == p:
+                    assert row[k] == b
+                elif p < 300:
+                    assert row[k] + q >= 0 and row[k] < 0
+
+
 # ---------------------------------------------------------------- table modes and root renumbering
 def test_table_modes_agree_and_root():
     for p, root in [(17, 0), (17, 5), (100, 99), (1000, 123), (1025, 7)]:
