@@ -61,6 +61,9 @@ def _load():
             lib.oracle_checksum.argtypes = [i64, u64p]
             lib.oracle_schedule_batch.argtypes = [i32p, i32p, i32p, i64, ctypes.c_int32,
                                                   ctypes.c_int32, i32p, i32p]
+            lib.oracle_shift_rows.argtypes = [ctypes.c_int, i64, i64, i32p]
+            lib.oracle_simulate_broadcast.argtypes = [i64, i64, i64, i32p, i32p, i32p, u64p]
+            lib.oracle_simulate_reduce.argtypes = [i64, i64, i64, i32p, i32p, u64p, u64p, u64p]
             _lib = lib
     return _lib
 
@@ -215,3 +218,50 @@ def schedule_batch(p, rank, root, row_stride: int = 31, pad: int = PAD,
     if rc < 0:
         raise ValueError("bad query in batch")
     return recv, send
+
+
+def _u64(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))
+
+
+def shifted_table(p: int, n: int, root: int = 0, rank_begin: int = 0, rank_end: int | None = None):
+    """Algorithm 1's preamble applied to the tables: (x, recv, send) ready for n blocks."""
+    recv, send = schedule_table(p, root, rank_begin, rank_end)
+    q = q_of(p)
+    x = 0
+    if q > 0:
+        x = _load().oracle_shift_rows(q, n, recv.shape[0], _i32(recv))
+        _load().oracle_shift_rows(q, n, send.shape[0], _i32(send))
+        if x < 0:
+            raise ValueError("bad arguments")
+    return x, recv, send
+
+
+def simulate_broadcast(p: int, root: int, n: int, recv_tab, send_tab):
+    """Algorithm 1 by all processors on the given tables: (arrival[n][p] int32, stats[8] uint64)."""
+    q = q_of(p)
+    recv_tab = np.ascontiguousarray(recv_tab, dtype=np.int32).reshape(p, q)
+    send_tab = np.ascontiguousarray(send_tab, dtype=np.int32).reshape(p, q)
+    arrival = np.zeros((n, p), dtype=np.int32)
+    stats = np.zeros(8, dtype=np.uint64)
+    if _load().oracle_simulate_broadcast(p, root, n, _i32(recv_tab), _i32(send_tab), _i32(arrival),
+                                         _u64(stats)) < 0:
+        raise ValueError("bad arguments to simulate_broadcast")
+    return arrival, stats
+
+
+def simulate_reduce(p: int, root: int, n: int, recv_tab, send_tab, value):
+    """Observation 1.3's reduction (wrapping 64-bit sum) on the given tables.
+
+    value: [n][p] uint64 contributions (not modified).  Returns (result[n] uint64, stats[8] uint64).
+    """
+    q = q_of(p)
+    recv_tab = np.ascontiguousarray(recv_tab, dtype=np.int32).reshape(p, q)
+    send_tab = np.ascontiguousarray(send_tab, dtype=np.int32).reshape(p, q)
+    work = np.array(value, dtype=np.uint64, copy=True).reshape(n, p)
+    result = np.zeros(n, dtype=np.uint64)
+    stats = np.zeros(8, dtype=np.uint64)
+    if _load().oracle_simulate_reduce(p, root, n, _i32(recv_tab), _i32(send_tab), _u64(work), _u64(result),
+                                      _u64(stats)) < 0:
+        raise ValueError("bad arguments to simulate_reduce")
+    return result, stats

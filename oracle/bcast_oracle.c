@@ -501,3 +501,230 @@ int oracle_schedule_batch(const int32_t *p, const int32_t *rank, const int32_t *
     }
     return 0;
 }
+
+/*
+ * Algorithm 1's preamble for a whole table: the rows Broadcast() starts its
+ * communication loop with when n blocks are broadcast.  With
+ * x = (q - (n-1) mod q) mod q every entry has x subtracted, and the entries of
+ * the rounds i < x, which are virtual and already "done", have q added.
+ * In place on `rows` rows of q entries.
+ */
+int oracle_shift_rows(int q, int64_t n, int64_t rows, int32_t *tab)
+{
+    int64_t x, a;
+    int i;
+    if (q < 1 || n < 1 || rows < 0) return -1;
+    x = (q - (n - 1) % q) % q;
+    for (a = 0; a < rows; a++)
+        for (i = 0; i < q; i++) {
+            tab[a * q + i] = (int32_t)(tab[a * q + i] - x);
+            if (i < x) tab[a * q + i] += q;
+        }
+    return (int)x;
+}
+
+/*
+ * Algorithm 1 run by all p processors in lock-step on given schedule tables
+ * (rows indexed by actual rank, as oracle_schedule_table writes them), blocks
+ * moved by the rules the paper leaves to the Send||Recv operation: a negative
+ * block is neither sent nor received, a block above n-1 stands for n-1,
+ * nothing is sent to the root and the root receives nothing.
+ *
+ * Every processor keeps its own shifted copy of both rows (the preamble above)
+ * and adds q to an entry after each use, as printed.  A round has two halves:
+ * first every processor decides, from what it held BEFORE the round, what it
+ * puts on the wire; then every processor takes what its from-processor sent.
+ *
+ * arrival[b * p + a]: the communication round (counted from 1) in which
+ * processor a received block b; 0 for the root (it has the blocks from the
+ * start); -1 if it never arrived.  A block is delivered only if the sender
+ * sends exactly the block the receiver expects and held it before the round
+ * and the receiver does not hold it yet.
+ * stats[0] receiver expects a block, sender sends another one or nothing
+ * stats[1] matching block, but the sender did not hold it before the round
+ * stats[2] matching block that the receiver already holds
+ * stats[3] a block is sent to a processor (not the root) that expects nothing
+ * stats[4] (processor, block) pairs still missing after the last round
+ * stats[5] table entries outside [-q, q-1] (they count as "nothing" in every round)
+ * stats[6] blocks delivered
+ * stats[7] last round in which something was delivered
+ */
+int oracle_simulate_broadcast(int64_t p, int64_t root, int64_t n,
+                              const int32_t *recv_tab, const int32_t *send_tab,
+                              int32_t *arrival, uint64_t *stats)
+{
+    int q = oracle_q(p);
+    int64_t skip[ORACLE_MAXQ + 2];
+    int64_t x, i, a, b, rounds;
+    int64_t *rb, *sb, *wire;
+    unsigned char *rvalid, *svalid, *wire_held;
+    int k;
+    if (q < 0 || n < 1 || root < 0 || root >= p) return -1;
+    memset(stats, 0, 8 * sizeof(uint64_t));
+    for (b = 0; b < n; b++)
+        for (a = 0; a < p; a++) arrival[b * p + a] = (a == root) ? 0 : -1;
+    if (q == 0) return 0;
+    oracle_skips(p, skip);
+    rounds = n - 1 + q;
+    x = (q - (n - 1) % q) % q;
+    rb = (int64_t *)malloc((size_t)p * q * sizeof(int64_t));
+    sb = (int64_t *)malloc((size_t)p * q * sizeof(int64_t));
+    rvalid = (unsigned char *)malloc((size_t)p * q);
+    svalid = (unsigned char *)malloc((size_t)p * q);
+    wire = (int64_t *)malloc((size_t)p * sizeof(int64_t));
+    wire_held = (unsigned char *)malloc((size_t)p);
+    if (!rb || !sb || !rvalid || !svalid || !wire || !wire_held) {
+        free(rb); free(sb); free(rvalid); free(svalid); free(wire); free(wire_held);
+        return -2;
+    }
+    for (a = 0; a < p; a++)
+        for (i = 0; i < q; i++) {
+            int32_t rv = recv_tab[a * q + i], sv = send_tab[a * q + i];
+            rvalid[a * q + i] = (rv >= -q && rv <= q - 1);
+            svalid[a * q + i] = (sv >= -q && sv <= q - 1);
+            if (!rvalid[a * q + i]) stats[5]++;
+            if (!svalid[a * q + i]) stats[5]++;
+            rb[a * q + i] = (int64_t)rv - x;
+            sb[a * q + i] = (int64_t)sv - x;
+            if (i < x) { rb[a * q + i] += q; sb[a * q + i] += q; }
+        }
+    for (i = x; i < n + q - 1 + x; i++) {
+        int64_t round = i - x + 1;                 /* communication rounds counted from 1 */
+        k = (int)(i % q);
+        /* first half: what goes on the wire, from the state before the round */
+        for (a = 0; a < p; a++) {
+            int64_t t = (a + skip[k]) % p;
+            int64_t blk = sb[a * q + k];
+            wire[a] = -1;
+            wire_held[a] = 0;
+            if (svalid[a * q + k] && blk >= 0 && t != root) {
+                if (blk > n - 1) blk = n - 1;
+                wire[a] = blk;
+                wire_held[a] = (arrival[blk * p + a] >= 0);
+            }
+        }
+        /* second half: every processor but the root takes what its from-processor sent */
+        for (a = 0; a < p; a++) {
+            int64_t f = (a - skip[k] + p) % p;
+            int64_t want = rb[a * q + k];
+            if (a == root) continue;
+            if (!rvalid[a * q + k] || want < 0) want = -1;
+            else if (want > n - 1) want = n - 1;
+            if (want < 0) {
+                if (wire[f] >= 0) stats[3]++;
+            } else if (wire[f] != want) {
+                stats[0]++;
+            } else if (!wire_held[f]) {
+                stats[1]++;
+            } else if (arrival[want * p + a] >= 0) {
+                stats[2]++;
+            } else {
+                arrival[want * p + a] = (int32_t)round;
+                stats[6]++;
+                stats[7] = (uint64_t)round;
+            }
+        }
+        for (a = 0; a < p; a++) { sb[a * q + k] += q; rb[a * q + k] += q; }
+    }
+    (void)rounds;
+    for (b = 0; b < n; b++)
+        for (a = 0; a < p; a++)
+            if (arrival[b * p + a] < 0) stats[4]++;
+    free(rb); free(sb); free(rvalid); free(svalid); free(wire); free(wire_held);
+    return q;
+}
+
+/*
+ * The reduction of Observation 1 (item 3): Algorithm 1 with every communication
+ * reversed, rounds taken downwards from (n-1+q+x)-1 to x, and the received
+ * block combined into the processor's own partial result.  In the round that
+ * was broadcast round i, processor a sends its partial result of block
+ * recvblock[k] to its from-processor f and receives, from its to-processor t,
+ * a partial result of block sendblock[k], which it adds to its own.  The same
+ * exceptions, reversed: a negative block moves nothing, a block above n-1
+ * stands for n-1, the root sends nothing (it received nothing), and a
+ * processor whose to-processor is the root receives nothing.
+ *
+ * The operator here is the wrapping 64-bit sum; processor a contributes
+ * value[b * p + a] to block b (overwritten with the partial results).
+ * result[b]: the root's value of block b after the last round.
+ * A partial result is combined only if the receiver expects exactly the block
+ * the sender sends and has not passed its own partial result of it on yet.
+ * stats[0] receiver expects a block, sender sends another one or nothing
+ * stats[1] matching block, but the receiver has sent (or is sending) its partial result of it
+ * stats[2] a processor sends a block it has sent before
+ * stats[3] a block is sent to a processor that expects nothing
+ * stats[4] (non-root processor, block) pairs whose partial result was not sent exactly once
+ * stats[5] table entries outside [-q, q-1]
+ * stats[6] partial results combined
+ * stats[7] unused (0)
+ */
+int oracle_simulate_reduce(int64_t p, int64_t root, int64_t n,
+                           const int32_t *recv_tab, const int32_t *send_tab,
+                           uint64_t *value, uint64_t *result, uint64_t *stats)
+{
+    int q = oracle_q(p);
+    int64_t skip[ORACLE_MAXQ + 2];
+    int64_t x, i, a, b;
+    int64_t *wire;
+    uint64_t *wire_val;
+    int32_t *times_sent;
+    int k;
+    if (q < 0 || n < 1 || root < 0 || root >= p) return -1;
+    memset(stats, 0, 8 * sizeof(uint64_t));
+    if (q == 0) { for (b = 0; b < n; b++) result[b] = value[b]; return 0; }
+    oracle_skips(p, skip);
+    x = (q - (n - 1) % q) % q;
+    wire = (int64_t *)malloc((size_t)p * sizeof(int64_t));
+    wire_val = (uint64_t *)malloc((size_t)p * sizeof(uint64_t));
+    times_sent = (int32_t *)calloc((size_t)p * n, sizeof(int32_t));
+    if (!wire || !wire_val || !times_sent) { free(wire); free(wire_val); free(times_sent); return -2; }
+    for (a = 0; a < p; a++)
+        for (k = 0; k < q; k++) {
+            int32_t rv = recv_tab[a * q + k], sv = send_tab[a * q + k];
+            if (rv < -q || rv > q - 1) stats[5]++;
+            if (sv < -q || sv > q - 1) stats[5]++;
+        }
+    for (i = n + q - 1 + x - 1; i >= x; i--) {
+        int64_t phase = i / q;
+        k = (int)(i % q);
+        /* the entry Algorithm 1 uses in round i: shifted by -x and one q per phase (Theorem 1) */
+        for (a = 0; a < p; a++) {
+            int32_t rv = recv_tab[a * q + k];
+            int64_t blk = (int64_t)rv + phase * q - x;
+            wire[a] = -1;
+            if (a == root || rv < -q || rv > q - 1 || blk < 0) continue;
+            if (blk > n - 1) blk = n - 1;
+            wire[a] = blk;
+            wire_val[a] = value[blk * p + a];
+            if (times_sent[blk * p + a] > 0) stats[2]++;
+        }
+        for (a = 0; a < p; a++) {
+            int64_t t = (a + skip[k]) % p;
+            int32_t sv = send_tab[a * q + k];
+            int64_t want = (int64_t)sv + phase * q - x;
+            if (sv < -q || sv > q - 1 || want < 0 || t == root) want = -1;
+            else if (want > n - 1) want = n - 1;
+            if (want < 0) {
+                if (t != root && wire[t] >= 0) stats[3]++;
+            } else if (wire[t] != want) {
+                stats[0]++;
+            } else if (a != root && (times_sent[want * p + a] > 0 || wire[a] == want)) {
+                stats[1]++;                        /* it would never be passed on */
+            } else {
+                value[want * p + a] += wire_val[t];
+                stats[6]++;
+            }
+        }
+        /* the sends of this round are now in the past */
+        for (a = 0; a < p; a++)
+            if (wire[a] >= 0) times_sent[wire[a] * p + a]++;
+    }
+    for (b = 0; b < n; b++) {
+        result[b] = value[b * p + root];
+        for (a = 0; a < p; a++)
+            if (a != root && times_sent[b * p + a] != 1) stats[4]++;
+    }
+    free(wire); free(wire_val); free(times_sent);
+    return q;
+}

@@ -40,6 +40,17 @@ MUTANTS = [
     ("Algorithm 7: send rows from the to-side", "int64_t f = (j - c.skip[k] + p) % p;", "int64_t f = (j + c.skip[k]) % p;"),
     ("root renumbering", "int64_t r = (a - root + p) % p;\n                recvschedule_(&c, r, tmp, NULL);\n                for (k = 0; k < q; k++) recv_tab",
      "int64_t r = (a + root) % p;\n                recvschedule_(&c, r, tmp, NULL);\n                for (k = 0; k < q; k++) recv_tab"),
+    ("Algorithm 1's preamble: virtual rounds include x", "if (i < x) tab[a * q + i] += q;", "if (i <= x) tab[a * q + i] += q;"),
+    ("simulated broadcast: virtual rounds not moved to the next phase",
+     "if (i < x) { rb[a * q + i] += q; sb[a * q + i] += q; }", ";"),
+    ("simulated broadcast: rounds counted from the virtual ones", "int64_t round = i - x + 1;", "int64_t round = i + 1;"),
+    ("simulated broadcast: sender's holdings not checked", "} else if (!wire_held[f]) {", "} else if (0) {"),
+    ("simulated reduction: partial results travel the broadcast's way",
+     "int64_t t = (a + skip[k]) % p;\n            int32_t sv", "int64_t t = (a - skip[k] + p) % p;\n            int32_t sv"),
+    ("simulated reduction: received value replaces the partial result", "value[want * p + a] += wire_val[t];",
+     "value[want * p + a] = wire_val[t];"),
+    ("simulated reduction: rounds not reversed", "for (i = n + q - 1 + x - 1; i >= x; i--) {",
+     "for (i = x; i < n + q - 1 + x; i++) {"),
 ]
 
 

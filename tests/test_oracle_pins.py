@@ -482,3 +482,146 @@ def test_allbroadcast_simulation():
                 for r, j, blk in arrivals:
                     held[r, j, blk] = True
             assert held.all(), (p, n)
+
+
+# ---------------------------------------------------------------- Algorithm 1 by all processors; its reversal
+def _arrival_by_theorem1(p, n, root, recv):
+    """Theorem 1 read backwards: processor a receives block recv[k] + q*floor(i/q) - x in round i = x + j
+    whatever the others do, so the round each block arrives in follows from a's own row."""
+    q = recv.shape[1]
+    arrival = np.full((n, p), -1, dtype=np.int64)
+    arrival[:, root] = 0
+    if q == 0:
+        return arrival
+    x = (q - (n - 1) % q) % q
+    for a in range(p):
+        if a == root:
+            continue
+        for j in range(n - 1 + q):
+            i = x + j
+            raw = int(recv[a, i % q]) + q * (i // q) - x
+            if raw >= 0:
+                blk = min(raw, n - 1)
+                assert arrival[blk, a] == -1, "a block would arrive twice"
+                arrival[blk, a] = j + 1
+    return arrival
+
+
+def test_simulated_broadcast_of_correct_tables():
+    for p in list(range(1, 41)) + [63, 64, 65, 100]:
+        q = oracle.q_of(p)
+        for n in [1, 2, 3, q, q + 1, 2 * q + 3, 11]:
+            if n < 1:
+                continue
+            for root in {0, p // 3, p - 1}:
+                recv, send = oracle.schedule_table(p, root)
+                arrival, stats = oracle.simulate_broadcast(p, root, n, recv, send)
+                assert list(stats[:6]) == [0] * 6, (p, n, root, stats)
+                assert stats[6] == (p - 1) * n
+                assert stats[7] == (n - 1 + q if p > 1 else 0)        # the optimal number of rounds, all used
+                assert (arrival == _arrival_by_theorem1(p, n, root, recv)).all()
+                assert arrival.max() <= n - 1 + q and (arrival[:, root] == 0).all()
+
+
+def test_simulated_broadcast_power_of_two_single_block():
+    # one block on p = 2^q processors: processor r is reached in round floor(log2 r) + 1
+    for q in range(1, 9):
+        p = 1 << q
+        recv, send = oracle.schedule_table(p)
+        arrival, stats = oracle.simulate_broadcast(p, 0, 1, recv, send)
+        assert list(arrival[0]) == [0] + [r.bit_length() for r in range(1, p)]
+        assert stats[7] == q
+
+
+def test_simulated_broadcast_agrees_with_the_brute_force_checker():
+    for p, n, root in [(17, 8, 5), (33, 13, 32), (57, 6, 0), (1000, 8, 0)]:
+        recv, send = oracle.schedule_table(p, root)
+        q = recv.shape[1]
+
+        def rounds_of(rrow, srow):
+            _, k, rr, sr = oracle.broadcast_rounds(q, n, rrow, srow)
+            return k, rr, sr
+
+        res = simulate(p, n, root, oracle.skips(p), recv, send, rounds_of)
+        arrival, stats = oracle.simulate_broadcast(p, root, n, recv, send)
+        assert ((arrival >= 0).T == res["held"]).all()
+        assert int(arrival.max()) == res["done_round"]
+
+
+def test_simulated_broadcast_notices_damaged_tables():
+    p, n, root = 37, 9, 4
+    recv, send = oracle.schedule_table(p, root)
+    q = recv.shape[1]
+    # a send entry changed: the receiver no longer gets what it expects
+    s2 = send.copy(); s2[10, 2] = s2[10, 2] - 1 if s2[10, 2] > -q else s2[10, 2] + 1
+    arrival, stats = oracle.simulate_broadcast(p, root, n, recv, s2)
+    assert stats[0] + stats[3] > 0 and stats[4] > 0 and (arrival < 0).any()
+    # an entry out of range is counted and moves nothing
+    r2 = recv.copy(); r2[20, 1] = q
+    _, stats = oracle.simulate_broadcast(p, root, n, r2, send)
+    assert stats[5] == 1 and stats[3] + stats[0] > 0
+    # a processor and its from-processor agree on a block the sender does not hold yet: both tables of
+    # round 0 say "block of the next phase"
+    a = (root + 5) % p
+    f = (a - 1) % p
+    r3, s3 = recv.copy(), send.copy()
+    r3[a, 0] = q - 1; s3[f, 0] = q - 1
+    _, stats = oracle.simulate_broadcast(p, root, n, r3, s3)
+    assert stats[1] > 0
+    # the tables of another root
+    _, stats = oracle.simulate_broadcast(p, (root + 1) % p, n, recv, send)
+    assert sum(int(v) for v in stats[:5]) > 0
+
+
+def test_shifted_tables_are_algorithm_1s_starting_rows():
+    for p in [2, 9, 17, 18, 100]:
+        q = oracle.q_of(p)
+        recv, send = oracle.schedule_table(p)
+        for n in range(1, 3 * q + 2):
+            x, srecv, ssend = oracle.shifted_table(p, n)
+            assert (n - 1 + x) % q == 0 and 0 <= x < q
+            for a in [0, 1, p // 2, p - 1]:
+                # the first use of entry k in the printed loop reads exactly the shifted entry
+                _, k, rr, sr = oracle.broadcast_rounds(q, n, recv[a], send[a])
+                seen = set()
+                for j in range(min(n - 1 + q, q)):
+                    if int(k[j]) not in seen:
+                        seen.add(int(k[j]))
+                        assert rr[j] == srecv[a, k[j]] and sr[j] == ssend[a, k[j]]
+            # entries of rounds before x belong to the next phase
+            assert ((srecv - recv) == np.where(np.arange(q) < x, q - x, -x)).all()
+
+
+def _contributions(p, n, seed):
+    return np.random.default_rng(seed).integers(0, 2 ** 63, size=(n, p), dtype=np.uint64)
+
+
+def test_simulated_reduction_gives_the_sum():
+    for p in list(range(1, 34)) + [63, 64, 65, 100]:
+        q = oracle.q_of(p)
+        for n in [1, 2, q, q + 1, 2 * q + 3]:
+            if n < 1:
+                continue
+            for root in {0, p // 3, p - 1}:
+                recv, send = oracle.schedule_table(p, root)
+                value = _contributions(p, n, p * 131 + n)
+                result, stats = oracle.simulate_reduce(p, root, n, recv, send, value)
+                with np.errstate(over="ignore"):
+                    want = value.sum(axis=1, dtype=np.uint64)           # the definition of the reduction
+                assert (result == want).all(), (p, n, root)
+                assert list(stats[:6]) == [0] * 6, (p, n, root, stats)
+                assert stats[6] == (p - 1) * n                          # every partial result moved exactly once
+
+
+def test_simulated_reduction_notices_damaged_tables():
+    p, n, root = 37, 9, 4
+    recv, send = oracle.schedule_table(p, root)
+    q = recv.shape[1]
+    value = _contributions(p, n, 7)
+    with np.errstate(over="ignore"):
+        want = value.sum(axis=1, dtype=np.uint64)
+    r2 = recv.copy(); r2[10, 2] = r2[10, 2] - 1 if r2[10, 2] > -q else r2[10, 2] + 1
+    result, stats = oracle.simulate_reduce(p, root, n, r2, send, value)
+    assert sum(int(v) for v in stats[:5]) > 0 and (result != want).any()
+    result, stats = oracle.simulate_reduce(p, (root + 1) % p, n, recv, send, value)
+    assert sum(int(v) for v in stats[:5]) > 0
