@@ -85,6 +85,20 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
                    int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);
 
 /*
+ * bcast_schedule with the rows already prepared for n blocks, i.e. after the
+ * preamble of Algorithm 1: with x = (q - (n-1) mod q) mod q virtual rounds in
+ * front, every entry has x subtracted, and the entries of the rounds k < x
+ * (already "done" when communication starts) have q added, so that the loop of
+ * Algorithm 1 can use entry k = i mod q as it is and add q after each use.
+ * Entries lie in [-2q+1, 2q-2].  n >= 1 (BCAST_EINVAL_N otherwise); everything
+ * else as for bcast_schedule.  n - 1 a multiple of q gives x = 0 and the
+ * unshifted tables.  Returns q; x is what bcast_round reports as -shift for
+ * round j = 0.
+ */
+int bcast_schedule_shifted(int32_t p, int32_t root, int64_t n, int64_t rank_begin, int64_t rank_end,
+                           int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);
+
+/*
  * The schedule part of Algorithm 7 (all-broadcast, Appendix A) for one processor
  * `rank`: with every processor j as root in turn, row j - root_begin of
  * recvblocks_dev receives recvschedule((rank - j + p) mod p) and the same row of
@@ -191,6 +205,82 @@ int bcast_verify_sweep(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
  */
 int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev,
                               uint32_t *fail_counts_dev, void *cuda_stream);
+
+/*
+ * Algorithm 1 carried out by all p processors at once on given tables (Section 2;
+ * the exceptions are those the paper leaves to its Send||Recv operation): in
+ * communication round j = 0 .. n-2+q, with i = x + j, k = i mod q, processor a
+ * sends block sendblock[a][k] + q*floor(i/q) - x to (a + skip[k]) mod p and
+ * receives block recvblock[a][k] + q*floor(i/q) - x from (a - skip[k]) mod p; a
+ * negative block moves nothing, a block above n-1 stands for block n-1, nothing
+ * is sent to the root and the root receives nothing.  A stronger check than the
+ * conditions of bcast_verify_sweep: the blocks really travel.
+ *
+ * recvblock_dev, sendblock_dev: device int32 tables [p][q] of ALL actual ranks
+ * as bcast_schedule(p, root, 0, p, ...) writes them (not modified; NULL allowed
+ * only for p = 1).
+ * arrival_dev: device int32 [n][p], written by the call: arrival[b*p + a] is the
+ * round, counted from 1, in which processor a received block b; 0 for the root;
+ * -1 if the block never arrived.  A block is delivered only when the sender
+ * sends exactly the block the receiver expects, held it before the round, and
+ * the receiver does not hold it yet.
+ * stats_dev: device uint64[8], 8-byte aligned, zeroed and filled by the call:
+ *   [0] receiver expects a block, its from-processor sends another one or nothing
+ *   [1] matching block that the sender did not hold before the round
+ *   [2] matching block that the receiver already holds
+ *   [3] a block sent to a processor (not the root) that expects nothing
+ *   [4] (processor, block) pairs still missing after the last round
+ *   [5] table entries outside [-q, q-1] (they move nothing in any round)
+ *   [6] blocks delivered                    (correct tables: (p-1)*n)
+ *   [7] last round that delivered a block   (correct tables: n-1+q)
+ * Correct tables give zeros in [0..5].
+ * scratch_dev: device memory, 16-byte aligned, at least
+ * bcast_simulate_scratch_bytes(p, n, 0) bytes; it receives round-major byte
+ * copies of the tables.  Contents after the call are unspecified.
+ * Launches n-1+q small kernels on cuda_stream, asynchronously.  Returns q.
+ * Limits: n < 2^31 - 64; n * p int32 cells must fit the caller's memory.
+ */
+int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction);
+int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
+                             const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                             int32_t *arrival_dev, uint64_t *stats_dev,
+                             void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
+
+/*
+ * The reduction of Observation 1, item 3: the rounds of Algorithm 1 taken from
+ * the last to the first with every communication reversed.  In the round that
+ * is broadcast round i, processor a sends its partial result of block
+ * recvblock[a][k] + q*floor(i/q) - x to its from-processor (a - skip[k]) mod p
+ * and receives a partial result of block sendblock[a][k] + q*floor(i/q) - x from
+ * its to-processor (a + skip[k]) mod p, which it combines with its own.  The
+ * root sends nothing, a processor whose to-processor is the root receives
+ * nothing; negative blocks and blocks above n-1 as in the broadcast.  The
+ * operator is the wrapping sum of uint64.
+ *
+ * value_dev: device uint64 [n][p], 8-byte aligned: value[b*p + a] is processor
+ * a's contribution to block b on entry and its partial result on return.
+ * result_dev: device uint64 [n]: the root's value of each block after the last
+ * round (correct tables: the sum over all processors).
+ * A partial result is combined only when the receiver expects exactly the block
+ * the sender sends and has not sent (and is not sending) its own partial result
+ * of that block.
+ * stats_dev: device uint64[8], zeroed and filled by the call:
+ *   [0] receiver expects a block, its to-processor sends another one or nothing
+ *   [1] matching block whose partial result the receiver has already passed on
+ *   [2] a processor sends a block it has sent before
+ *   [3] a block sent to a processor that expects nothing
+ *   [4] (non-root processor, block) pairs not sent exactly once
+ *   [5] table entries outside [-q, q-1]
+ *   [6] partial results combined            (correct tables: (p-1)*n)
+ *   [7] unused, 0
+ * scratch_dev: at least bcast_simulate_scratch_bytes(p, n, 1) bytes, 16-byte
+ * aligned.  Tables, limits, asynchrony and return value as for
+ * bcast_simulate_broadcast; two launches per round.
+ */
+int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
+                          const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                          uint64_t *value_dev, uint64_t *result_dev, uint64_t *stats_dev,
+                          void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
 
 /*
  * Algorithm 1's use of a schedule row, O(1) per round.  For n >= 1 blocks and

@@ -46,6 +46,11 @@ def _load():
         lib.bcast_verify_sweep_scratch_bytes.restype = i64
         lib.bcast_verify_sweep.argtypes = [i32, i32, vp, vp, vp, i64, vp]
         lib.bcast_verify_sweep_static.argtypes = [i32, i32, vp, vp, vp]
+        lib.bcast_schedule_shifted.argtypes = [i32, i32, i64, i64, i64, vp, vp, vp]
+        lib.bcast_simulate_scratch_bytes.argtypes = [i32, i64, ctypes.c_int]
+        lib.bcast_simulate_scratch_bytes.restype = i64
+        lib.bcast_simulate_broadcast.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, i64, vp]
+        lib.bcast_simulate_reduce.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_round.argtypes = [i32, i64, i64, ctypes.POINTER(i32), ctypes.POINTER(i64)]
         lib.bcast_round_block.argtypes = [i32, i64, i64, vp]
         lib.bcast_round_block.restype = i64
@@ -116,6 +121,33 @@ def bcast_schedule(p: int, root: int, rank_begin: int, rank_end: int, recvblock,
     """Fill int32 device tensors [rank_end-rank_begin, q]; either may be None. Returns q."""
     return _check(_load().bcast_schedule(p, root, rank_begin, rank_end, _ptr(recvblock), _ptr(sendblock),
                                          _stream(stream)))
+
+
+def bcast_schedule_shifted(p: int, root: int, n: int, rank_begin: int, rank_end: int, recvblock, sendblock,
+                           stream=None) -> int:
+    """bcast_schedule with Algorithm 1's preamble for n blocks applied to every row. Returns q."""
+    return _check(_load().bcast_schedule_shifted(p, root, n, rank_begin, rank_end, _ptr(recvblock),
+                                                 _ptr(sendblock), _stream(stream)))
+
+
+def bcast_simulate_scratch_bytes(p: int, n: int, reduction: bool = False) -> int:
+    return _check(_load().bcast_simulate_scratch_bytes(p, n, 1 if reduction else 0))
+
+
+def bcast_simulate_broadcast(p: int, root: int, n: int, recvblock, sendblock, arrival, stats, scratch,
+                             stream=None) -> int:
+    """Algorithm 1 by all processors on device tables [p, q]: fills arrival [n, p] int32 and stats [8] uint64."""
+    nbytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    return _check(_load().bcast_simulate_broadcast(p, root, n, _ptr(recvblock), _ptr(sendblock), _ptr(arrival),
+                                                   _ptr(stats), _ptr(scratch), nbytes, _stream(stream)))
+
+
+def bcast_simulate_reduce(p: int, root: int, n: int, recvblock, sendblock, value, result, stats, scratch,
+                          stream=None) -> int:
+    """The reversed rounds as a wrapping-sum reduction of value [n, p] (uint64 bits); result [n], stats [8]."""
+    nbytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
+    return _check(_load().bcast_simulate_reduce(p, root, n, _ptr(recvblock), _ptr(sendblock), _ptr(value),
+                                                _ptr(result), _ptr(stats), _ptr(scratch), nbytes, _stream(stream)))
 
 
 def bcast_allbroadcast_schedule(p: int, rank: int, root_begin: int, root_end: int, recvblocks, sendblocks,
@@ -206,3 +238,26 @@ def verify_sweep(p_lo: int, p_hi: int, device="cuda"):
     scratch = torch.empty(bcast_verify_sweep_scratch_bytes(p_lo, p_hi), dtype=torch.uint8, device=device)
     bcast_verify_sweep(p_lo, p_hi, checksum, fails, scratch)
     return checksum, fails
+
+
+def simulate_broadcast(p: int, root: int, n: int, recvblock, sendblock):
+    """Allocate buffers and run Algorithm 1 on the tables; returns (arrival [n, p] int32, stats [8] as int64 bits)."""
+    import torch
+    dev = recvblock.device if recvblock is not None else "cuda"
+    arrival = torch.empty((n, p), dtype=torch.int32, device=dev)
+    stats = torch.empty(8, dtype=torch.int64, device=dev)
+    scratch = torch.empty(bcast_simulate_scratch_bytes(p, n), dtype=torch.uint8, device=dev)
+    bcast_simulate_broadcast(p, root, n, recvblock, sendblock, arrival, stats, scratch)
+    return arrival, stats
+
+
+def simulate_reduce(p: int, root: int, n: int, recvblock, sendblock, value):
+    """Allocate buffers and run the reduction on a copy of value [n, p] (int64 tensor holding uint64 bits);
+    returns (result [n], stats [8]) as int64 bit patterns."""
+    import torch
+    work = value.clone()
+    result = torch.empty(n, dtype=torch.int64, device=value.device)
+    stats = torch.empty(8, dtype=torch.int64, device=value.device)
+    scratch = torch.empty(bcast_simulate_scratch_bytes(p, n, True), dtype=torch.uint8, device=value.device)
+    bcast_simulate_reduce(p, root, n, recvblock, sendblock, work, result, stats, scratch)
+    return result, stats

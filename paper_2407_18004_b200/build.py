@@ -6,13 +6,15 @@ import subprocess
 import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = [os.path.join(_HERE, "csrc", "bcast_sched.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", "bcast_sched.cu"),
+           os.path.join(_HERE, "csrc", "bcast_simulate.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "schedule_core.cuh"),
+           os.path.join(_HERE, "csrc", "schedule_fast.cuh"),
            os.path.join(os.path.dirname(_HERE), "include", "bcast_sched.h")]
 LIBRARY = os.path.join(_HERE, "libbcast_sched.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--extended-lambda", "-shared", "-Xcompiler", "-fPIC", "-cudart", "shared"]
+              "--extended-lambda", "-Xcompiler", "-fPIC", "-cudart", "shared"]
 
 
 def needs_build() -> bool:
@@ -26,9 +28,20 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or needs_build():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIBRARY + ".tmp.%d" % os.getpid()
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
-        subprocess.check_call(cmd)
-        os.replace(tmp, LIBRARY)
+        flags = NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else [])
+        # one object per source, compiled side by side, then one link
+        objects = [tmp + ".%d.o" % i for i in range(len(SOURCES))]
+        procs = [subprocess.Popen([nvcc] + flags + ["-c", "-o", obj, src]) for src, obj in zip(SOURCES, objects)]
+        codes = [proc.wait() for proc in procs]
+        try:
+            if any(codes):
+                raise subprocess.CalledProcessError(max(codes), nvcc)
+            subprocess.check_call([nvcc] + NVCC_FLAGS + ["-shared", "-o", tmp] + objects)
+            os.replace(tmp, LIBRARY)
+        finally:
+            for obj in objects:
+                if os.path.exists(obj):
+                    os.remove(obj)
     return LIBRARY
 
 

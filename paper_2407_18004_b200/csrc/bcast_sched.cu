@@ -115,6 +115,26 @@ __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t 
     for (int i = done + lane; i < n_entries; i += kGroup) __stcs(out + i, (int)stage_bytes[i]);
 }
 
+// Algorithm 1's preamble applied to a staged byte tile in place: entry k of every row gets
+// -x, and +q on top when k < x (the rounds before x are virtual, their entries belong to the
+// next phase).  The tile starts at a row boundary, so byte e is column e mod Q; the shifted
+// values stay within [-2q+1, 2q-2] and fit a byte.  Called by the whole block.
+template <int Q>
+__device__ __forceinline__ void shift_tile(uint32_t *stage_words, int n_entries, int x)
+{
+    const int n_words = (n_entries + 3) >> 2;
+    for (int i = threadIdx.x; i < n_words; i += kThreads) {
+        const int c0 = (4 * i) % Q;
+        uint32_t add = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = (c0 + j) % Q;
+            add |= (uint32_t)((c < x ? Q - x : -x) & 0xff) << (8 * j);
+        }
+        stage_words[i] = __vadd4(stage_words[i], add);
+    }
+}
+
 // ------------------------------------------------------------------ all ranks of one p
 // Work the closed-form pass leaves behind, collected per tile of kThreads consecutive ranks.
 //
@@ -301,7 +321,7 @@ __global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
 schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t anchor,
                       uint32_t row_begin, uint32_t n_ranks, int descending, int tiles_per_block,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
-                      int recv_vec_ok, int send_vec_ok)
+                      int recv_vec_ok, int send_vec_ok, int shift_x)
 {
     typedef typename WalkInt<Q>::type Int;
     __shared__ uint32_t stage[2][(kThreads * Q + 15) / 16 * 4];   // byte tiles, kThreads rows of Q entries
@@ -361,6 +381,11 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         __syncthreads();
         if (queue.n_search + queue.n_copy > 0) {           // the same for every thread
             drain_queue(g, queue, tile, ns);
+            __syncthreads();
+        }
+        if (shift_x != 0) {                                // rows as Algorithm 1 starts with them for n blocks
+            if (want_recv) shift_tile<Q>(stage[0], (int)rows * Q, shift_x);
+            if (want_send) shift_tile<Q>(stage[1], (int)rows * Q, shift_x);
             __syncthreads();
         }
         const size_t base = (size_t)first * (size_t)Q;
@@ -729,7 +754,7 @@ int bcast_skips(int32_t p, int32_t *skip_host)
 
 // Launch of the table kernel for n_rows output rows starting at global row index row_begin.
 static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int64_t n_rows, int descending,
-                        int32_t *recv_dev, int32_t *send_dev, void *cuda_stream)
+                        int32_t *recv_dev, int32_t *send_dev, void *cuda_stream, int shift_x = 0)
 {
     const int sms = sm_count();
     if (sms <= 0) return BCAST_ECUDA;
@@ -748,7 +773,7 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     case N:                                                                                               \
         schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)anchor,       \
             (uint32_t)row_begin, (uint32_t)n_rows, descending, (int)tiles_per_block, recv_dev, send_dev,  \
-            recv_vec, send_vec);                                                                          \
+            recv_vec, send_vec, shift_x);                                                                 \
         break;
         BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6) BCAST_CASE(7)
         BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12) BCAST_CASE(13)
@@ -774,6 +799,22 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
     if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
     if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
     return launch_table(p, q, root, rank_begin, n_ranks, 0, recvblock_dev, sendblock_dev, cuda_stream);
+}
+
+int bcast_schedule_shifted(int32_t p, int32_t root, int64_t n, int64_t rank_begin, int64_t rank_end,
+                           int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
+    if (n < 1) return BCAST_EINVAL_N;
+    if (rank_begin < 0 || rank_begin > rank_end || rank_end > p) return BCAST_EINVAL_RANGE;
+    const int q = host_q(p);
+    const int64_t n_ranks = rank_end - rank_begin;
+    if (q == 0 || n_ranks == 0) return q;
+    if (recvblock_dev == nullptr && sendblock_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)recvblock_dev & 3u) || ((uintptr_t)sendblock_dev & 3u)) return BCAST_EALIGN;
+    const int x = (int)((q - (n - 1) % q) % q);
+    return launch_table(p, q, root, rank_begin, n_ranks, 0, recvblock_dev, sendblock_dev, cuda_stream, x);
 }
 
 int bcast_allbroadcast_schedule(int32_t p, int32_t rank, int64_t root_begin, int64_t root_end,

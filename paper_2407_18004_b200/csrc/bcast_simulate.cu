@@ -1,0 +1,368 @@
+// Device-side use of schedule tables: Algorithm 1 of arXiv 2407.18004 run by all p
+// processors at once, round by round, on tables in device memory (bcast_simulate_broadcast),
+// and the same rounds reversed as a reduction (Observation 1, item 3: bcast_simulate_reduce).
+// See include/bcast_sched.h for the contracts.
+//
+// Layout and launch shape
+//   * The int32 tables [p][q] are first turned into round-major byte tables [q][P]
+//     (P = p rounded up to 128) in the caller's scratch: a round then reads one byte per
+//     processor from each table, consecutive processors from consecutive addresses, and the
+//     2q*P bytes stay in L2 over the n-1+q rounds.  Entries outside [-q, q-1] are counted
+//     and stored as kInvalid, which moves nothing in any round.
+//   * One thread per processor, one launch per round (two for the reduction: everybody
+//     sends, then everybody receives), all on the caller's stream.  Nothing waits on
+//     another block inside a launch.
+//   * Broadcast state is arrival[b][a], the round in which processor a got block b.  A
+//     sender "held the block before the round" iff its arrival is in [0, round); a value
+//     written during the round is >= round, so concurrent readers decide the same way
+//     whether or not they see it: one buffer, no race in the outcome.
+//   * Reduction state is value[b][a] plus a saturating count sent[b][a]; the messages of a
+//     round go through wire arrays (block, value) written by the send launch and read by
+//     the receive launch.
+//   * Counters are summed per warp with redux and added to the 64-bit statistics with one
+//     atomic per warp and counter that is not zero.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bcast_sched.h"
+
+namespace bcast_sim {
+
+constexpr int kThreads = 256;
+constexpr int8_t kInvalid = -128;
+constexpr int64_t kHeaderBytes = 256;
+
+__host__ __device__ inline int64_t padded(int64_t p) { return (p + 127) / 128 * 128; }
+
+static int host_q(int64_t p)
+{
+    int q = 0;
+    while (((int64_t)1 << q) < p) ++q;
+    return q;
+}
+
+__device__ __forceinline__ void add_stat(unsigned long long *stats, int index, unsigned int mine)
+{
+    const unsigned int total = __reduce_add_sync(0xffffffffu, mine);
+    if (total != 0u && (threadIdx.x & 31) == 0) atomicAdd(stats + index, (unsigned long long)total);
+}
+
+// int32 [p][q] -> int8 [q][P], both tables (blockIdx.y), a tile of kThreads processors per block.
+__global__ void __launch_bounds__(kThreads)
+transpose_tables_kernel(const int32_t *__restrict__ recv_tab, const int32_t *__restrict__ send_tab,
+                        int8_t *__restrict__ recv_t, int8_t *__restrict__ send_t,
+                        uint32_t p, int q, size_t P, unsigned long long *stats)
+{
+    __shared__ int8_t tile[kThreads * 33];                 // rows of q <= 31 bytes, 33 apart
+    const int32_t *in = blockIdx.y == 0 ? recv_tab : send_tab;
+    int8_t *out = blockIdx.y == 0 ? recv_t : send_t;
+    const uint32_t first = blockIdx.x * kThreads;
+    const uint32_t rows = min((uint32_t)kThreads, p - first);
+    const int n_entries = (int)rows * q;
+    const int32_t *src = in + (size_t)first * q;
+    unsigned int bad = 0;
+    for (int i = threadIdx.x; i < n_entries; i += kThreads) {
+        const int v = src[i];
+        const bool ok = v >= -q && v <= q - 1;
+        bad += ok ? 0u : 1u;
+        const int row = i / q;
+        tile[row * 33 + (i - row * q)] = ok ? (int8_t)v : kInvalid;
+    }
+    __syncthreads();
+    if (threadIdx.x < rows)
+        for (int k = 0; k < q; ++k) out[(size_t)k * P + first + threadIdx.x] = tile[threadIdx.x * 33 + k];
+    add_stat(stats, 5, bad);
+}
+
+__global__ void __launch_bounds__(kThreads)
+init_arrival_kernel(int32_t *__restrict__ arrival, uint32_t p, uint32_t root)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    if (a < p) arrival[(size_t)blockIdx.y * p + a] = a == root ? 0 : -1;
+}
+
+// Block of a table entry in a round: entry + shift, nothing (-1) when negative or invalid,
+// n-1 when above it.
+__device__ __forceinline__ int64_t block_of(int8_t entry, int64_t shift, int64_t n)
+{
+    if (entry == kInvalid) return -1;
+    const int64_t raw = (int64_t)entry + shift;
+    if (raw < 0) return -1;
+    return raw > n - 1 ? n - 1 : raw;
+}
+
+// One communication round of Algorithm 1 for every processor: skip index k (the rows of the
+// byte tables passed in), blocks = entry + shift, `round` counted from 1.
+__global__ void __launch_bounds__(kThreads)
+broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
+                       int32_t *arrival, uint32_t p, uint32_t root, int64_t n, uint32_t skip_k,
+                       int64_t shift, int32_t round, unsigned long long *stats)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
+    if (a < p && a != root) {
+        const uint32_t f = a >= skip_k ? a - skip_k : a + (p - skip_k);     // from-processor
+        const int64_t want = block_of(recv_k[a], shift, n);
+        // f's to-processor is a, which is not the root, so f's send is not suppressed
+        const int64_t sent = block_of(send_k[f], shift, n);
+        if (want < 0) {
+            if (sent >= 0) c3 = 1;
+        } else if (sent != want) {
+            c0 = 1;
+        } else {
+            const int32_t at_f = arrival[(size_t)want * p + f];
+            const int32_t at_a = arrival[(size_t)want * p + a];
+            if (!(at_f >= 0 && at_f < round)) c1 = 1;                        // not held before the round
+            else if (at_a >= 0) c2 = 1;
+            else { arrival[(size_t)want * p + a] = round; c6 = 1; }
+        }
+    }
+    add_stat(stats, 0, c0);
+    add_stat(stats, 1, c1);
+    add_stat(stats, 2, c2);
+    add_stat(stats, 3, c3);
+    add_stat(stats, 6, c6);
+    if (__any_sync(0xffffffffu, c6 != 0u) && (threadIdx.x & 31) == 0)
+        atomicMax(stats + 7, (unsigned long long)round);
+}
+
+__global__ void __launch_bounds__(kThreads)
+count_missing_kernel(const int32_t *__restrict__ arrival, size_t cells, unsigned long long *stats)
+{
+    unsigned int missing = 0;
+    for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < cells; i += (size_t)gridDim.x * kThreads)
+        missing += arrival[i] < 0 ? 1u : 0u;
+    add_stat(stats, 4, missing);
+}
+
+// ------------------------------------------------------------------ reduction (reversed rounds)
+// First half of a reduction round: processor a puts its partial result of the block it
+// RECEIVED in the corresponding broadcast round on the wire (the root sends nothing).
+__global__ void __launch_bounds__(kThreads)
+reduce_send_kernel(const int8_t *__restrict__ recv_k, const uint64_t *__restrict__ value,
+                   const uint8_t *__restrict__ sent, int32_t *__restrict__ wire_block,
+                   uint64_t *__restrict__ wire_value, uint32_t p, uint32_t root, int64_t n,
+                   int64_t shift, unsigned long long *stats)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    unsigned int c2 = 0;
+    if (a < p) {
+        const int64_t blk = a == root ? -1 : block_of(recv_k[a], shift, n);
+        wire_block[a] = (int32_t)blk;                      // n - 1 < 2^31 is checked on the host
+        if (blk >= 0) {
+            wire_value[a] = value[(size_t)blk * p + a];
+            if (sent[(size_t)blk * p + a] > 0) c2 = 1;
+        }
+    }
+    add_stat(stats, 2, c2);
+}
+
+// Second half: processor a takes, from its to-processor t, a partial result of the block it
+// SENT to t in the corresponding broadcast round and adds it to its own; then it notes its
+// own send of this round as done.
+__global__ void __launch_bounds__(kThreads)
+reduce_recv_kernel(const int8_t *__restrict__ send_k, uint64_t *value, uint8_t *sent,
+                   const int32_t *__restrict__ wire_block, const uint64_t *__restrict__ wire_value,
+                   uint32_t p, uint32_t root, int64_t n, uint32_t skip_k, int64_t shift,
+                   unsigned long long *stats)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    unsigned int c0 = 0, c1 = 0, c3 = 0, c6 = 0;
+    if (a < p) {
+        uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
+        if (t >= p) t -= p;
+        const int64_t want = t == root ? -1 : block_of(send_k[a], shift, n);
+        const int64_t mine = wire_block[a];
+        const int64_t got = t == root ? -1 : (int64_t)wire_block[t];
+        if (want < 0) {
+            if (got >= 0) c3 = 1;
+        } else if (got != want) {
+            c0 = 1;
+        } else if (a != root && (sent[(size_t)want * p + a] > 0 || mine == want)) {
+            c1 = 1;                                        // it would never be passed on
+        } else {
+            value[(size_t)want * p + a] += wire_value[t];
+            c6 = 1;
+        }
+        if (mine >= 0) {
+            const uint8_t before = sent[(size_t)mine * p + a];
+            if (before < 2) sent[(size_t)mine * p + a] = before + 1;
+        }
+    }
+    add_stat(stats, 0, c0);
+    add_stat(stats, 1, c1);
+    add_stat(stats, 3, c3);
+    add_stat(stats, 6, c6);
+}
+
+__global__ void __launch_bounds__(kThreads)
+reduce_finish_kernel(const uint64_t *__restrict__ value, const uint8_t *__restrict__ sent,
+                     uint64_t *__restrict__ result, uint32_t p, uint32_t root, unsigned long long *stats)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const size_t b = blockIdx.y;
+    unsigned int c4 = 0;
+    if (a < p) {
+        if (a == root) result[b] = value[b * p + a];
+        else if (sent[b * p + a] != 1) c4 = 1;
+    }
+    add_stat(stats, 4, c4);
+}
+
+__global__ void copy_row_kernel(const uint64_t *__restrict__ value, uint64_t *__restrict__ result, int64_t n)
+{
+    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < n) result[b] = value[b];
+}
+
+struct Plan {
+    int q;
+    int64_t P;
+    int64_t x;
+    uint32_t skip[33];
+};
+
+static Plan make_plan(int32_t p, int64_t n)
+{
+    Plan plan = {};
+    plan.q = host_q(p);
+    plan.P = padded(p);
+    plan.x = plan.q > 0 ? (plan.q - (n - 1) % plan.q) % plan.q : 0;
+    int64_t s = p;
+    plan.skip[plan.q] = (uint32_t)p;
+    for (int k = plan.q; k > 0; --k) {
+        s = s - s / 2;
+        plan.skip[k - 1] = (uint32_t)s;
+    }
+    return plan;
+}
+
+static int check_common(int32_t p, int32_t root, int64_t n, const void *recv, const void *send,
+                        const void *state, const void *stats)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (root < 0 || root >= p) return BCAST_EINVAL_ROOT;
+    if (n < 1 || n > (int64_t)0x7fffffff - 64) return BCAST_EINVAL_N;
+    if (state == nullptr || stats == nullptr) return BCAST_ENULL;
+    if (p > 1 && (recv == nullptr || send == nullptr)) return BCAST_ENULL;
+    if (((uintptr_t)recv & 3u) || ((uintptr_t)send & 3u) || ((uintptr_t)stats & 7u)) return BCAST_EALIGN;
+    return BCAST_OK;
+}
+
+}  // namespace bcast_sim
+
+using namespace bcast_sim;
+
+extern "C" {
+
+int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (n < 1) return BCAST_EINVAL_N;
+    const int q = host_q(p);
+    const int64_t P = padded(p);
+    int64_t bytes = kHeaderBytes + 2 * (int64_t)q * P;
+    if (reduction) bytes += 8 * P + 4 * P + n * (int64_t)p;        // wire values, wire blocks, sent counts
+    return bytes;
+}
+
+int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
+                             const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                             int32_t *arrival_dev, uint64_t *stats_dev,
+                             void *scratch_dev, int64_t scratch_bytes, void *cuda_stream)
+{
+    const int rc = check_common(p, root, n, recvblock_dev, sendblock_dev, arrival_dev, stats_dev);
+    if (rc != BCAST_OK) return rc;
+    if ((uintptr_t)arrival_dev & 3u) return BCAST_EALIGN;
+    const Plan plan = make_plan(p, n);
+    const int q = plan.q;
+    if (q > 0) {
+        if (scratch_dev == nullptr) return BCAST_ENULL;
+        if ((uintptr_t)scratch_dev & 15u) return BCAST_EALIGN;
+        if (scratch_bytes < bcast_simulate_scratch_bytes(p, n, 0)) return BCAST_ESCRATCH;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long *stats = reinterpret_cast<unsigned long long *>(stats_dev);
+    if (cudaMemsetAsync(stats_dev, 0, 8 * sizeof(uint64_t), stream) != cudaSuccess) return BCAST_ECUDA;
+    const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
+    // blocks of the arrival table go in slices of at most 65535 (the grid's y limit)
+    for (int64_t b0 = 0; b0 < n; b0 += 65535) {
+        const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
+        init_arrival_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(arrival_dev + (size_t)b0 * p, (uint32_t)p,
+                                                                       (uint32_t)root);
+    }
+    if (q > 0) {
+        int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
+        int8_t *send_t = recv_t + (size_t)q * plan.P;
+        transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
+            recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
+        const int64_t rounds = n - 1 + q;
+        for (int64_t j = 0; j < rounds; ++j) {
+            const int64_t i = plan.x + j;
+            const int k = (int)(i % q);
+            const int64_t shift = (i / q) * q - plan.x;            // Theorem 1
+            broadcast_round_kernel<<<blocks, kThreads, 0, stream>>>(
+                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, (uint32_t)p,
+                (uint32_t)root, n, plan.skip[k], shift, (int32_t)(j + 1), stats);
+        }
+    }
+    const size_t cells = (size_t)n * (size_t)p;
+    const size_t want_blocks = (cells + kThreads - 1) / kThreads;
+    count_missing_kernel<<<(unsigned int)(want_blocks < 148 * 16 ? want_blocks : 148 * 16), kThreads, 0, stream>>>(
+        arrival_dev, cells, stats);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return q;
+}
+
+int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
+                          const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                          uint64_t *value_dev, uint64_t *result_dev, uint64_t *stats_dev,
+                          void *scratch_dev, int64_t scratch_bytes, void *cuda_stream)
+{
+    const int rc = check_common(p, root, n, recvblock_dev, sendblock_dev, value_dev, stats_dev);
+    if (rc != BCAST_OK) return rc;
+    if (result_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)value_dev & 7u) || ((uintptr_t)result_dev & 7u)) return BCAST_EALIGN;
+    const Plan plan = make_plan(p, n);
+    const int q = plan.q;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long *stats = reinterpret_cast<unsigned long long *>(stats_dev);
+    if (cudaMemsetAsync(stats_dev, 0, 8 * sizeof(uint64_t), stream) != cudaSuccess) return BCAST_ECUDA;
+    if (q == 0) {                                                  // one processor: its values are the result
+        copy_row_kernel<<<(unsigned int)((n + 255) / 256), 256, 0, stream>>>(value_dev, result_dev, n);
+        return cudaGetLastError() == cudaSuccess ? 0 : BCAST_ECUDA;
+    }
+    if (scratch_dev == nullptr) return BCAST_ENULL;
+    if ((uintptr_t)scratch_dev & 15u) return BCAST_EALIGN;
+    if (scratch_bytes < bcast_simulate_scratch_bytes(p, n, 1)) return BCAST_ESCRATCH;
+    int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
+    int8_t *send_t = recv_t + (size_t)q * plan.P;
+    uint64_t *wire_value = reinterpret_cast<uint64_t *>(send_t + (size_t)q * plan.P);
+    int32_t *wire_block = reinterpret_cast<int32_t *>(wire_value + plan.P);
+    uint8_t *sent = reinterpret_cast<uint8_t *>(wire_block + plan.P);
+    if (cudaMemsetAsync(sent, 0, (size_t)n * (size_t)p, stream) != cudaSuccess) return BCAST_ECUDA;
+    const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
+    transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
+        recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
+    const int64_t rounds = n - 1 + q;
+    for (int64_t j = rounds - 1; j >= 0; --j) {                    // the broadcast's rounds, last one first
+        const int64_t i = plan.x + j;
+        const int k = (int)(i % q);
+        const int64_t shift = (i / q) * q - plan.x;
+        reduce_send_kernel<<<blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, value_dev, sent,
+                                                            wire_block, wire_value, (uint32_t)p, (uint32_t)root,
+                                                            n, shift, stats);
+        reduce_recv_kernel<<<blocks, kThreads, 0, stream>>>(send_t + (size_t)k * plan.P, value_dev, sent,
+                                                            wire_block, wire_value, (uint32_t)p, (uint32_t)root,
+                                                            n, plan.skip[k], shift, stats);
+    }
+    for (int64_t b0 = 0; b0 < n; b0 += 65535) {
+        const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
+        reduce_finish_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(
+            value_dev + (size_t)b0 * p, sent + (size_t)b0 * p, result_dev + b0, (uint32_t)p, (uint32_t)root, stats);
+    }
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return q;
+}
+
+}  // extern "C"

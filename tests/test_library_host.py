@@ -23,7 +23,8 @@ def test_library_exports_every_declared_symbol():
     lib = ctypes.CDLL(bs.library_path())
     names = declared_functions()
     assert {"bcast_q", "bcast_skips", "bcast_schedule", "bcast_schedule_host", "bcast_schedule_batch",
-            "bcast_allbroadcast_schedule", "bcast_verify_sweep_static",
+            "bcast_allbroadcast_schedule", "bcast_verify_sweep_static", "bcast_schedule_shifted",
+            "bcast_simulate_scratch_bytes", "bcast_simulate_broadcast", "bcast_simulate_reduce",
             "bcast_verify_sweep", "bcast_verify_sweep_scratch_bytes", "bcast_round", "bcast_round_block",
             "bcast_strerror"} <= set(names)
     for name in names:
