@@ -12,6 +12,12 @@ Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent
 replica of the workload (the path has no exchange step), timed as the maximum
 over ranks.  `--impl reference` times the CPU oracle on a bounded sample of the
 same workload on the host cores.
+
+Other workloads of the same library, each with its own metric (`--mode`):
+allbroadcast (Algorithm 7's tables), shifted (tables after Algorithm 1's
+preamble), batch (2^24 independent queries), sweep (fused verification of every
+p in [2, 65536]), simulate / reduce (Algorithm 1 and its reversal run by all
+processors on device tables).
 """
 from __future__ import annotations
 
@@ -63,9 +69,10 @@ def kernel_source_hash() -> str:
     return h.hexdigest()
 
 
-def recorded_traffic(kernel: str, p: int):
-    """dram read+write bytes per launch from profiles/dram_traffic.txt, or None when the sources changed since."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+def recorded_traffic(kernel: str, p, filename: str = "dram_traffic.txt"):
+    """Sum of the two counters of one launch recorded in profiles/<filename> (DRAM bytes read + written, or
+    warp instructions + 0), or None when the sources changed since they were taken."""
+    path = os.path.join(ROOT, "profiles", filename)
     if not os.path.exists(path):
         return None
     sha = kernel_source_hash()
@@ -134,7 +141,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle_sample(p: int, budget_ranks: int, mode: str = "broadcast"):
+def time_oracle_sample(p: int, budget_ranks: int, mode: str = "broadcast", blocks: int = 0):
     """The oracle as it stands on a window of rows of the same workload (single thread)."""
     import oracle
     oracle.build()
@@ -142,6 +149,8 @@ def time_oracle_sample(p: int, budget_ranks: int, mode: str = "broadcast"):
     t0 = time.perf_counter()
     if mode == "allbroadcast":
         oracle.allbroadcast_schedule(p, p // 3, 0, hi)
+    elif mode == "shifted":
+        oracle.shifted_table(p, blocks, 0, 0, hi)
     else:
         oracle.schedule_table(p, 0, 0, hi)
     dt = time.perf_counter() - t0
@@ -153,7 +162,10 @@ def time_oracle_sample(p: int, budget_ranks: int, mode: str = "broadcast"):
     return hi / dt, dt, sample
 
 
-def workload_label(mode: str, p: int, q: int) -> str:
+def workload_label(mode: str, p: int, q: int, blocks: int = 0) -> str:
+    if mode == "shifted":
+        return ("all ranks of p=%d (q=%d), root 0, tables with Algorithm 1's preamble for n=%d blocks applied"
+                % (p, q, blocks))
     if mode == "allbroadcast":
         return ("Algorithm 7 tables of processor %d for all roots of p=%d (q=%d), recvblocks+sendblocks int32"
                 % (p // 3, p, q))
@@ -179,6 +191,8 @@ def run_reference(args):
     def ref_step():
         if args.mode == "allbroadcast":
             oracle.allbroadcast_schedule(p, p // 3, 0, per_step)
+        elif args.mode == "shifted":
+            oracle.shifted_table(p, args.blocks, 0, 0, per_step)
         else:
             oracle.schedule_table(p, 0, 0, per_step)
 
@@ -196,7 +210,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
         "data": "synthetic",
-        "config": {"workload": workload_label(args.mode, p, q), "sampled": True},
+        "config": {"workload": workload_label(args.mode, p, q, args.blocks), "sampled": True},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -233,6 +247,8 @@ def run_ours(args):
         bs.bcast_skips(p)
         if args.mode == "allbroadcast":
             bs.bcast_allbroadcast_schedule(p, p // 3, 0, p, recv, send, stream)
+        elif args.mode == "shifted":
+            bs.bcast_schedule_shifted(p, 0, args.blocks, 0, p, recv, send, stream)
         else:
             bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
 
@@ -320,7 +336,7 @@ def run_ours(args):
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        v, dt, sample = time_oracle_sample(p, oracle_sample_size(p), args.mode)
+        v, dt, sample = time_oracle_sample(p, oracle_sample_size(p), args.mode, args.blocks)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                         "seconds": dt, "host_cores_available": os.cpu_count()}
 
@@ -328,7 +344,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": workload_label(args.mode, p, q),
+        "config": {"workload": workload_label(args.mode, p, q, args.blocks),
                    "bytes_per_step": table_bytes, "replicas": world,
                    "l2": "tables larger than L2" if flush is None else "L2 flushed between steps"},
         "entries_per_s": value * 2 * q,
@@ -349,6 +365,354 @@ def run_ours(args):
     return 0
 
 
+# ---------------------------------------------------------------------------------------------
+# The other workloads: each a dict with its metric, one device step, the oracle on a bounded
+# sample, and an end-to-end step that moves its inputs and results over PCIe.
+OTHER_MODES = ("batch", "sweep", "simulate", "reduce")
+ISSUE_PEAK_GINST = 148 * 4 * 1.965         # warp instructions per ns at one per scheduler and clock: 148 SMs x 4 x 1.965 GHz
+
+
+def build_other(args, torch, bs):
+    import numpy as np
+    from paper_2407_18004_b200 import workloads
+    stream = torch.cuda.current_stream()
+    mode = args.mode
+    if mode == "batch":
+        nq = args.queries
+        hp, hr, ho = workloads.query_batch(nq, seed=0)
+        pin = [torch.from_numpy(a).pin_memory() for a in (hp, hr, ho)]
+        dp, dr, do = [t.cuda() for t in pin]
+        recv = torch.empty((nq, 31), dtype=torch.int32, device="cuda")
+        send = torch.empty((nq, 31), dtype=torch.int32, device="cuda")
+        bad = torch.zeros(1, dtype=torch.int32, device="cuda")
+        host_out = {}
+
+        def step():
+            bs.bcast_schedule_batch(dp, dr, do, 31, recv, send, bad, stream)
+
+        def e2e_step():
+            if not host_out:
+                host_out["r"] = torch.empty((nq, 31), dtype=torch.int32, pin_memory=True)
+                host_out["s"] = torch.empty((nq, 31), dtype=torch.int32, pin_memory=True)
+            for d, h in zip((dp, dr, do), pin):
+                d.copy_(h, non_blocking=True)
+            step()
+            host_out["r"].copy_(recv, non_blocking=True)
+            host_out["s"].copy_(send, non_blocking=True)
+
+        def oracle_sample():
+            import oracle
+            m = min(nq, 2 ** 19)
+            t0 = time.perf_counter()
+            oracle.schedule_batch(hp[:m], hr[:m], ho[:m], 31)
+            return m, time.perf_counter() - t0, ("the first %d queries: receive row by Algorithm 5, send row by "
+                                                 "definition (q receive schedules)" % m)
+
+        return dict(label="%d queries, p log-uniform in [2, 2^31-1], rank and root uniform, seed 0, rows padded to 31"
+                          % nq, metric="schedule_queries_per_s", unit="queries/s", units=nq,
+                    bytes=nq * (2 * 31 * 4 + 12), step=step, launches=1, kernel="schedule_batch_kernel",
+                    bound="alu", e2e=e2e_step, h2d=12 * nq, d2h=2 * 31 * 4 * nq, oracle=oracle_sample,
+                    extra=lambda: {"bad_queries": int(bad.item())})
+    if mode == "sweep":
+        lo, hi = args.sweep_lo, args.sweep_hi
+        checksum = torch.zeros(hi - lo + 1, dtype=torch.int64, device="cuda")
+        fails = torch.zeros(8, dtype=torch.int32, device="cuda")
+        scratch = torch.empty(bs.bcast_verify_sweep_scratch_bytes(lo, hi), dtype=torch.uint8, device="cuda")
+        units = sum(range(lo, hi + 1))
+        host = {}
+
+        def step():
+            bs.bcast_verify_sweep(lo, hi, checksum, fails, scratch, stream)
+
+        def e2e_step():
+            if not host:
+                host["c"] = torch.empty(hi - lo + 1, dtype=torch.int64, pin_memory=True)
+                host["f"] = torch.empty(8, dtype=torch.int32, pin_memory=True)
+            step()
+            host["c"].copy_(checksum, non_blocking=True)
+            host["f"].copy_(fails, non_blocking=True)
+
+        def oracle_sample():
+            import oracle
+            ps = list(range(hi, lo - 1, -(hi - lo) // 96))[:96]
+            t0 = time.perf_counter()
+            for pp in ps:
+                oracle.checksum(pp)
+            return sum(ps), time.perf_counter() - t0, ("checksums of %d values of p spread evenly over [%d, %d] "
+                                                       "(tables by Algorithm 5 and a gather, no condition checks)"
+                                                       % (len(ps), lo, hi))
+
+        return dict(label="every p in [%d, %d], all ranks, root 0: tables built and checked on the device, one "
+                          "checksum per p" % (lo, hi), metric="verified_rank_schedules_per_s", unit="rank-schedules/s",
+                    units=units, bytes=8 * (hi - lo + 1), step=step, launches=2, kernel="verify_sweep_kernel",
+                    bound="alu", e2e=e2e_step, h2d=0, d2h=8 * (hi - lo + 1) + 32, oracle=oracle_sample,
+                    extra=lambda: {"fail_counts": fails.tolist()})
+    # simulate / reduce
+    p = workload_of(args.workload)
+    q = bs.bcast_q(p)
+    n = args.blocks
+    rounds = n - 1 + q
+    recv = torch.empty((p, q), dtype=torch.int32, device="cuda")
+    send = torch.empty((p, q), dtype=torch.int32, device="cuda")
+    bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
+    stats = torch.zeros(8, dtype=torch.int64, device="cuda")
+    scratch = torch.empty(bs.bcast_simulate_scratch_bytes(p, n, mode == "reduce"), dtype=torch.uint8, device="cuda")
+    host = {}
+    small_p = min(p, 2 ** 16 + 1)
+    if mode == "simulate":
+        arrival = torch.empty((n, p), dtype=torch.int32, device="cuda")
+
+        def step():
+            bs.bcast_simulate_broadcast(p, 0, n, recv, send, arrival, stats, scratch, stream)
+
+        def e2e_step():
+            if not host:
+                host["s"] = torch.empty(8, dtype=torch.int64, pin_memory=True)
+            bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
+            step()
+            host["s"].copy_(stats, non_blocking=True)
+
+        def oracle_sample():
+            import oracle
+            r, s = oracle.schedule_table(small_p, 0)
+            t0 = time.perf_counter()
+            oracle.simulate_broadcast(small_p, 0, n, r, s)
+            return (small_p - 1) * n, time.perf_counter() - t0, ("the same %d blocks on p=%d processors (tables given)"
+                                                                 % (n, small_p))
+
+        # tables turned into bytes (8q read, 2q written per processor), arrival table set and counted (4 B per
+        # cell each), and per round and processor two table bytes, two arrival reads and one arrival write
+        nbytes = p * (10 * q + 8 * n + rounds * 14)
+        return dict(label="Algorithm 1 by all processors of p=%d (q=%d), n=%d blocks, %d rounds, tables on the device"
+                          % (p, q, n, rounds), metric="simulated_block_deliveries_per_s", unit="blocks/s",
+                    units=(p - 1) * n, bytes=nbytes, step=step, launches=rounds + 3, kernel="broadcast_round_kernel",
+                    bound="hbm", e2e=e2e_step, h2d=0, d2h=64, oracle=oracle_sample,
+                    extra=lambda: {"stats": stats.tolist()})
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(0)
+    contrib = torch.randint(0, 2 ** 62, (n, p), dtype=torch.int64, device="cuda", generator=gen)
+    value = torch.empty_like(contrib)
+    result = torch.empty(n, dtype=torch.int64, device="cuda")
+
+    def step():
+        value.copy_(contrib)
+        bs.bcast_simulate_reduce(p, 0, n, recv, send, value, result, stats, scratch, stream)
+
+    def e2e_step():
+        if not host:
+            host["s"] = torch.empty(8, dtype=torch.int64, pin_memory=True)
+            host["r"] = torch.empty(n, dtype=torch.int64, pin_memory=True)
+        bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
+        step()
+        host["s"].copy_(stats, non_blocking=True)
+        host["r"].copy_(result, non_blocking=True)
+
+    def oracle_sample():
+        import numpy as np
+        import oracle
+        r, s = oracle.schedule_table(small_p, 0)
+        v = np.random.default_rng(0).integers(0, 2 ** 62, size=(n, small_p), dtype=np.uint64)
+        t0 = time.perf_counter()
+        oracle.simulate_reduce(small_p, 0, n, r, s, v)
+        return (small_p - 1) * n, time.perf_counter() - t0, ("the same %d blocks on p=%d processors (tables given)"
+                                                             % (n, small_p))
+
+    # contributions copied in (16 B per cell), sent counts cleared and read (2 B per cell), byte tables, and per
+    # round and processor: two table bytes, wire block and value written and read, one value read, one value
+    # read-modify-write, sent count read twice and written once
+    nbytes = p * (10 * q + 18 * n + rounds * (2 + 24 + 8 + 16 + 3))
+    return dict(label="Observation 1.3's reduction by all processors of p=%d (q=%d), n=%d blocks, %d rounds"
+                      % (p, q, n, rounds), metric="simulated_partial_results_per_s", unit="blocks/s",
+                units=(p - 1) * n, bytes=nbytes, step=step, launches=2 * rounds + 4, kernel="reduce_recv_kernel",
+                bound="hbm", e2e=e2e_step, h2d=0, d2h=64 + 8 * n, oracle=oracle_sample,
+                extra=lambda: {"stats": stats.tolist()})
+
+
+def run_other(args):
+    if args.impl == "reference":
+        return run_other_reference(args)
+    import torch
+    import torch.distributed as dist
+    import paper_2407_18004_b200 as bs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the schedule library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = build_other(args, torch, bs)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, flush_between):
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        barrier()
+        for i in range(steps):
+            if flush_between:
+                flush.zero_()
+            starts[i].record(stream)
+            fn()
+            stops[i].record(stream)
+        barrier()
+        return [a.elapsed_time(b) for a, b in zip(starts, stops)]
+
+    for _ in range(max(args.warmup, 3)):
+        wl["step"]()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.15)
+    t0 = time.time()
+    per_step_ms = timed(wl["step"], args.steps, True)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    total_ms = sum(per_step_ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * wl["units"] * args.steps / (total_ms * 1e-3)
+
+    e2e = None
+    if not args.no_e2e:
+        wl["e2e"]()
+        torch.cuda.synchronize()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        e2e_ms = sum(timed(wl["e2e"], e2e_steps, False))
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * wl["units"] * e2e_steps / (e2e_ms * 1e-3), "unit": wl["unit"],
+               "h2d_bytes_per_step": wl["h2d"], "d2h_bytes_per_step": wl["d2h"], "steps": e2e_steps,
+               "ms_per_step": e2e_ms / e2e_steps}
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    mean_ms = statistics.mean(per_step_ms)
+    if wl["bound"] == "hbm":
+        peak, peak_src = measured_peaks()
+        achieved = wl["bytes"] / (mean_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": recorded_traffic(wl["kernel"], args.mode), "peak_source": peak_src,
+                    "kernel": wl["kernel"], "bytes_per_step": wl["bytes"],
+                    "note": "algorithmic bytes of the whole step over the step's time (many short launches)"}
+    else:
+        # bound by instruction issue: warp instructions of one launch (recorded from ncu while the sources
+        # are unchanged) over its time, against one instruction per scheduler and clock
+        insts = recorded_traffic(wl["kernel"], args.mode, "warp_instructions.txt")
+        achieved = insts / (mean_ms * 1e-3) / 1e9 if insts else None
+        roofline = {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
+                    "frac": achieved / ISSUE_PEAK_GINST if achieved else None, "traffic": None,
+                    "peak_source": "148 SMs x 4 schedulers x 1.965 GHz, one warp instruction per scheduler and clock",
+                    "kernel": wl["kernel"], "warp_instructions_per_launch": insts,
+                    "hbm_write_gbs": wl["bytes"] / (mean_ms * 1e-3) / 1e9}
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        units, dt, sample = wl["oracle"]()
+        cpu_baseline = {"value": units / dt, "unit": wl["unit"], "cores": 1, "kind": "oracle", "sample": sample,
+                        "seconds": dt, "host_cores_available": os.cpu_count()}
+    line = {
+        "metric": wl["metric"], "value": value, "unit": wl["unit"], "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": wl["label"], "bytes_per_step": wl["bytes"], "replicas": world,
+                   "l2": "L2 flushed between steps"},
+        "ms_per_step_min": min(per_step_ms), "ms_per_step_median": statistics.median(per_step_ms),
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+        "gpu_launches": args.steps * wl["launches"], "clocks": clocks,
+    }
+    line.update(wl["extra"]())
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def run_other_reference(args):
+    """The oracle's leg of the other workloads: its bounded sample, once per step."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    import oracle
+    oracle.build()
+
+    wl = reference_sample(args)
+    for _ in range(args.warmup):
+        wl()
+    units = 0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        u, _, sample = wl()
+        units += u
+    dt = time.perf_counter() - t0
+    metric, unit = {"batch": ("schedule_queries_per_s", "queries/s"),
+                    "sweep": ("verified_rank_schedules_per_s", "rank-schedules/s"),
+                    "simulate": ("simulated_block_deliveries_per_s", "blocks/s"),
+                    "reduce": ("simulated_partial_results_per_s", "blocks/s")}[args.mode]
+    value = units / dt
+    print(json.dumps({
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": args.mode, "sampled": True},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+    return 0
+
+
+def reference_sample(args):
+    """One step of the oracle's leg for the other workloads (sized for a run of a few minutes in all):
+    a function returning (units processed, unused, description of the sample)."""
+    import numpy as np
+    import oracle
+    from paper_2407_18004_b200 import workloads
+    share = max(args.steps + args.warmup, 1)
+    if args.mode == "batch":
+        m = max(2 ** 19 // share, 1024)
+        hp, hr, ho = workloads.query_batch(m, seed=0)
+
+        def batch_step():
+            oracle.schedule_batch(hp, hr, ho, 31)
+            return m, 0.0, "each step: %d queries of the seed-0 batch" % m
+        return batch_step
+    if args.mode == "sweep":
+        lo, hi = args.sweep_lo, args.sweep_hi
+        count = max(96 // share, 2)
+        ps = list(range(hi, lo - 1, -(hi - lo) // count))[:count]
+
+        def sweep_step():
+            for pp in ps:
+                oracle.checksum(pp)
+            return sum(ps), 0.0, "each step: checksums of p in %s" % ps
+        return sweep_step
+    p = min(workload_of(args.workload), 2 ** 16 + 1)
+    n = args.blocks
+    r, s = oracle.schedule_table(p, 0)
+    v = np.random.default_rng(0).integers(0, 2 ** 62, size=(n, p), dtype=np.uint64)
+
+    def simulate_step():
+        if args.mode == "simulate":
+            oracle.simulate_broadcast(p, 0, n, r, s)
+        else:
+            oracle.simulate_reduce(p, 0, n, r, s, v)
+        return (p - 1) * n, 0.0, "each step: %d blocks on p=%d processors" % (n, p)
+    return simulate_step
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -356,13 +720,25 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="p=2^27-1")
-    ap.add_argument("--mode", default="broadcast", choices=["broadcast", "allbroadcast"],
-                    help="broadcast: tables of all ranks for one root; allbroadcast: Algorithm 7's tables of one "
-                         "processor for all roots (no host-table leg)")
+    ap.add_argument("--mode", default="broadcast",
+                    choices=["broadcast", "allbroadcast", "shifted", "batch", "sweep", "simulate", "reduce"],
+                    help="broadcast: tables of all ranks for one root (the default, headline workload); "
+                         "allbroadcast: Algorithm 7's tables of one processor for all roots; shifted: tables with "
+                         "Algorithm 1's preamble for --blocks blocks; batch: 2^24 random (p, rank, root) queries; "
+                         "sweep: fused verification of every p in [2, 65536]; simulate / reduce: Algorithm 1 and "
+                         "its reversal run by all processors of --workload (default p=2^20+1) with --blocks blocks")
+    ap.add_argument("--blocks", type=int, default=64, help="n, the number of blocks (shifted, simulate, reduce)")
+    ap.add_argument("--queries", type=int, default=2 ** 24, help="number of queries (batch)")
+    ap.add_argument("--sweep-lo", type=int, default=2, help="first p of the sweep")
+    ap.add_argument("--sweep-hi", type=int, default=65536, help="last p of the sweep")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.mode in OTHER_MODES:
+        if args.workload == "p=2^27-1":
+            args.workload = "p=2^20+1"                     # the processors that simulate / reduce run on
+        return run_other(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -115,24 +115,52 @@ __device__ __forceinline__ void flush_tile(const uint32_t *stage_words, int32_t 
     for (int i = done + lane; i < n_entries; i += kGroup) __stcs(out + i, (int)stage_bytes[i]);
 }
 
-// Algorithm 1's preamble applied to a staged byte tile in place: entry k of every row gets
-// -x, and +q on top when k < x (the rounds before x are virtual, their entries belong to the
-// next phase).  The tile starts at a row boundary, so byte e is column e mod Q; the shifted
-// values stay within [-2q+1, 2q-2] and fit a byte.  Called by the whole block.
+// Algorithm 1's preamble for n blocks, applied while a tile is streamed out: entry k of every
+// row gets -x, and +q on top when k < x (the rounds before x are virtual, their entries
+// belong to the next phase).  The tile starts at a row boundary, so staged byte e is column
+// e mod Q.  shift_words[c] holds the four byte-wise addends for a word whose first byte is
+// column c; the sums stay within [-2q+1, 2q-2] and fit a byte.
 template <int Q>
-__device__ __forceinline__ void shift_tile(uint32_t *stage_words, int n_entries, int x)
+__device__ __forceinline__ void fill_shift_words(uint32_t *shift_words, int x)
 {
-    const int n_words = (n_entries + 3) >> 2;
-    for (int i = threadIdx.x; i < n_words; i += kThreads) {
-        const int c0 = (4 * i) % Q;
+    if (threadIdx.x < Q) {
         uint32_t add = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int c = (c0 + j) % Q;
+            const int c = ((int)threadIdx.x + j) % Q;
             add |= (uint32_t)((c < x ? Q - x : -x) & 0xff) << (8 * j);
         }
-        stage_words[i] = __vadd4(stage_words[i], add);
+        shift_words[threadIdx.x] = add;
     }
+}
+
+// Four byte sums without carries between the bytes.
+__device__ __forceinline__ uint32_t add_bytes(uint32_t a, uint32_t b)
+{
+    return ((a & 0x7f7f7f7fu) + (b & 0x7f7f7f7fu)) ^ ((a ^ b) & 0x80808080u);
+}
+
+// flush_tile by the whole block with the preamble's addends applied on the way out.
+template <int Q>
+__device__ __forceinline__ void flush_tile_shifted(const uint32_t *stage_words, const uint32_t *shift_words,
+                                                   int32_t *out, int n_entries, bool vec_ok, int x)
+{
+    const int8_t *stage_bytes = reinterpret_cast<const int8_t *>(stage_words);
+    int done = 0;
+    if (vec_ok) {
+        const int nvec = n_entries >> 2;
+        int4 *out4 = reinterpret_cast<int4 *>(out);
+        int c0 = (4 * (int)threadIdx.x) % Q;               // column of the word's first byte
+        constexpr int kStep = (4 * kThreads) % Q;
+        for (int i = threadIdx.x; i < nvec; i += kThreads) {
+            __stcs(out4 + i, widen4(add_bytes(stage_words[i], shift_words[c0])));
+            c0 += kStep;
+            if (c0 >= Q) c0 -= Q;
+        }
+        done = nvec << 2;
+    }
+    for (int i = done + (int)threadIdx.x; i < n_entries; i += kThreads)
+        __stcs(out + i, (int)stage_bytes[i] + (i % Q < x ? Q - x : -x));
 }
 
 // ------------------------------------------------------------------ all ranks of one p
@@ -328,6 +356,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
     __shared__ TileQueue queue;
     __shared__ LevelTables lookup;                         // the tables again, for per-lane indices
     __shared__ TileRuns<Int> runs[kWarpsPerBlock];         // descriptions of the next kWarpsPerBlock tiles
+    __shared__ uint32_t shift_words[32];                   // used only when shift_x != 0
     const Geometry g = make_geometry(p);
     const uint32_t n_tiles = (n_ranks + kThreads - 1u) / kThreads;
     const bool want_recv = recv_out != nullptr;
@@ -348,6 +377,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
     NoStats ns;
     if (threadIdx.x <= Q) lookup.skip[threadIdx.x] = tab.skip[threadIdx.x];
     if (threadIdx.x <= Q + 1) lookup.below[threadIdx.x] = tab.below[threadIdx.x];
+    if (shift_x != 0) fill_shift_words<Q>(shift_words, shift_x);
     __syncthreads();
 
     // This block's tiles: tiles_per_block (at most kWarpsPerBlock) consecutive ones.  Each warp first
@@ -383,12 +413,14 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             drain_queue(g, queue, tile, ns);
             __syncthreads();
         }
-        if (shift_x != 0) {                                // rows as Algorithm 1 starts with them for n blocks
-            if (want_recv) shift_tile<Q>(stage[0], (int)rows * Q, shift_x);
-            if (want_send) shift_tile<Q>(stage[1], (int)rows * Q, shift_x);
-            __syncthreads();
-        }
         const size_t base = (size_t)first * (size_t)Q;
+        if (shift_x != 0) {                                // rows as Algorithm 1 starts with them for n blocks
+            if (want_recv)
+                flush_tile_shifted<Q>(stage[0], shift_words, recv_out + base, (int)rows * Q, recv_vec_ok, shift_x);
+            if (want_send)
+                flush_tile_shifted<Q>(stage[1], shift_words, send_out + base, (int)rows * Q, send_vec_ok, shift_x);
+            continue;
+        }
         if (want_recv) flush_tile<kThreads>(stage[0], recv_out + base, (int)rows * Q, recv_vec_ok, threadIdx.x);
         if (want_send) flush_tile<kThreads>(stage[1], send_out + base, (int)rows * Q, send_vec_ok, threadIdx.x);
     }

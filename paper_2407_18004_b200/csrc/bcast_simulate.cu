@@ -19,8 +19,8 @@
 //   * Reduction state is value[b][a] plus a saturating count sent[b][a]; the messages of a
 //     round go through wire arrays (block, value) written by the send launch and read by
 //     the receive launch.
-//   * Counters are summed per warp with redux and added to the 64-bit statistics with one
-//     atomic per warp and counter that is not zero.
+//   * Counters are summed per warp with redux, per block in shared memory, and added to the
+//     64-bit statistics with one atomic per block and counter that is not zero.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -41,10 +41,33 @@ static int host_q(int64_t p)
     return q;
 }
 
-__device__ __forceinline__ void add_stat(unsigned long long *stats, int index, unsigned int mine)
+// Counters of one block: summed per warp with redux, per block in shared memory, and added
+// to the 64-bit statistics with one atomic per block and counter that is not zero (a round
+// of 2^20 processors would otherwise queue tens of thousands of atomics on one address).
+struct BlockStats {
+    unsigned int count[8];
+    unsigned int last_round;
+};
+
+__device__ __forceinline__ void stats_begin(BlockStats &bs)
+{
+    if (threadIdx.x < 8) bs.count[threadIdx.x] = 0u;
+    if (threadIdx.x == 8) bs.last_round = 0u;
+    __syncthreads();
+}
+
+__device__ __forceinline__ void add_stat(BlockStats &bs, int index, unsigned int mine)
 {
     const unsigned int total = __reduce_add_sync(0xffffffffu, mine);
-    if (total != 0u && (threadIdx.x & 31) == 0) atomicAdd(stats + index, (unsigned long long)total);
+    if (total != 0u && (threadIdx.x & 31) == 0) atomicAdd(&bs.count[index], total);
+}
+
+__device__ __forceinline__ void stats_end(BlockStats &bs, unsigned long long *stats)
+{
+    __syncthreads();
+    if (threadIdx.x < 8 && bs.count[threadIdx.x] != 0u)
+        atomicAdd(stats + threadIdx.x, (unsigned long long)bs.count[threadIdx.x]);
+    if (threadIdx.x == 8 && bs.last_round != 0u) atomicMax(stats + 7, (unsigned long long)bs.last_round);
 }
 
 // int32 [p][q] -> int8 [q][P], both tables (blockIdx.y), a tile of kThreads processors per block.
@@ -54,6 +77,8 @@ transpose_tables_kernel(const int32_t *__restrict__ recv_tab, const int32_t *__r
                         uint32_t p, int q, size_t P, unsigned long long *stats)
 {
     __shared__ int8_t tile[kThreads * 33];                 // rows of q <= 31 bytes, 33 apart
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     const int32_t *in = blockIdx.y == 0 ? recv_tab : send_tab;
     int8_t *out = blockIdx.y == 0 ? recv_t : send_t;
     const uint32_t first = blockIdx.x * kThreads;
@@ -71,7 +96,8 @@ transpose_tables_kernel(const int32_t *__restrict__ recv_tab, const int32_t *__r
     __syncthreads();
     if (threadIdx.x < rows)
         for (int k = 0; k < q; ++k) out[(size_t)k * P + first + threadIdx.x] = tile[threadIdx.x * 33 + k];
-    add_stat(stats, 5, bad);
+    add_stat(bstats, 5, bad);
+    stats_end(bstats, stats);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -98,6 +124,8 @@ broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restri
                        int32_t *arrival, uint32_t p, uint32_t root, int64_t n, uint32_t skip_k,
                        int64_t shift, int32_t round, unsigned long long *stats)
 {
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
     if (a < p && a != root) {
@@ -117,22 +145,25 @@ broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restri
             else { arrival[(size_t)want * p + a] = round; c6 = 1; }
         }
     }
-    add_stat(stats, 0, c0);
-    add_stat(stats, 1, c1);
-    add_stat(stats, 2, c2);
-    add_stat(stats, 3, c3);
-    add_stat(stats, 6, c6);
-    if (__any_sync(0xffffffffu, c6 != 0u) && (threadIdx.x & 31) == 0)
-        atomicMax(stats + 7, (unsigned long long)round);
+    add_stat(bstats, 0, c0);
+    add_stat(bstats, 1, c1);
+    add_stat(bstats, 2, c2);
+    add_stat(bstats, 3, c3);
+    add_stat(bstats, 6, c6);
+    if (__any_sync(0xffffffffu, c6 != 0u) && (threadIdx.x & 31) == 0) bstats.last_round = (unsigned int)round;
+    stats_end(bstats, stats);
 }
 
 __global__ void __launch_bounds__(kThreads)
 count_missing_kernel(const int32_t *__restrict__ arrival, size_t cells, unsigned long long *stats)
 {
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     unsigned int missing = 0;
     for (size_t i = (size_t)blockIdx.x * kThreads + threadIdx.x; i < cells; i += (size_t)gridDim.x * kThreads)
         missing += arrival[i] < 0 ? 1u : 0u;
-    add_stat(stats, 4, missing);
+    add_stat(bstats, 4, missing);
+    stats_end(bstats, stats);
 }
 
 // ------------------------------------------------------------------ reduction (reversed rounds)
@@ -144,6 +175,8 @@ reduce_send_kernel(const int8_t *__restrict__ recv_k, const uint64_t *__restrict
                    uint64_t *__restrict__ wire_value, uint32_t p, uint32_t root, int64_t n,
                    int64_t shift, unsigned long long *stats)
 {
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     unsigned int c2 = 0;
     if (a < p) {
@@ -154,7 +187,8 @@ reduce_send_kernel(const int8_t *__restrict__ recv_k, const uint64_t *__restrict
             if (sent[(size_t)blk * p + a] > 0) c2 = 1;
         }
     }
-    add_stat(stats, 2, c2);
+    add_stat(bstats, 2, c2);
+    stats_end(bstats, stats);
 }
 
 // Second half: processor a takes, from its to-processor t, a partial result of the block it
@@ -166,6 +200,8 @@ reduce_recv_kernel(const int8_t *__restrict__ send_k, uint64_t *value, uint8_t *
                    uint32_t p, uint32_t root, int64_t n, uint32_t skip_k, int64_t shift,
                    unsigned long long *stats)
 {
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     unsigned int c0 = 0, c1 = 0, c3 = 0, c6 = 0;
     if (a < p) {
@@ -189,16 +225,19 @@ reduce_recv_kernel(const int8_t *__restrict__ send_k, uint64_t *value, uint8_t *
             if (before < 2) sent[(size_t)mine * p + a] = before + 1;
         }
     }
-    add_stat(stats, 0, c0);
-    add_stat(stats, 1, c1);
-    add_stat(stats, 3, c3);
-    add_stat(stats, 6, c6);
+    add_stat(bstats, 0, c0);
+    add_stat(bstats, 1, c1);
+    add_stat(bstats, 3, c3);
+    add_stat(bstats, 6, c6);
+    stats_end(bstats, stats);
 }
 
 __global__ void __launch_bounds__(kThreads)
 reduce_finish_kernel(const uint64_t *__restrict__ value, const uint8_t *__restrict__ sent,
                      uint64_t *__restrict__ result, uint32_t p, uint32_t root, unsigned long long *stats)
 {
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     const size_t b = blockIdx.y;
     unsigned int c4 = 0;
@@ -206,7 +245,8 @@ reduce_finish_kernel(const uint64_t *__restrict__ value, const uint8_t *__restri
         if (a == root) result[b] = value[b * p + a];
         else if (sent[b * p + a] != 1) c4 = 1;
     }
-    add_stat(stats, 4, c4);
+    add_stat(bstats, 4, c4);
+    stats_end(bstats, stats);
 }
 
 __global__ void copy_row_kernel(const uint64_t *__restrict__ value, uint64_t *__restrict__ result, int64_t n)
