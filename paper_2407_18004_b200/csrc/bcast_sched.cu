@@ -14,8 +14,9 @@
 //                           then widens the tile to int32 and streams it out as one
 //                           contiguous run of 16-byte stores, so every store instruction
 //                           fills whole 32-byte sectors.
-//   schedule_batch_kernel   independent (p, rank, root) queries, one per thread: receive row by
-//                           the search, send row by Algorithm 6; rows padded to row_stride.
+//   schedule_batch_kernel   independent (p, rank, root) queries, one per thread, sorted by q within
+//                           a block so that a warp's lanes run loops of like length: receive row
+//                           by the search, send row by Algorithm 6; rows padded to row_stride.
 //   verify_sweep_kernel     persistent blocks pull values of p from a queue, build the tables
 //                           of one p in scratch memory with the table kernel's device
 //                           functions, then check the paper's correctness conditions against
@@ -427,78 +428,165 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
 }
 
 // ------------------------------------------------------------------ independent queries
+// A block takes kThreads consecutive queries.  Their q = ceil(log2 p) differ (1..31 for p drawn
+// log-uniformly), and every loop of the per-rank computation runs q or a few q times, so a
+// warp whose lanes hold unlike q idles most lanes most of the time.  The block therefore sorts
+// its queries by q (a counting sort in shared memory, longest first) and thread t computes the
+// query in position t of that order; rows are staged in shared memory at the query's own
+// position, so the output stays in the caller's order.
+constexpr int kBatchItems = 4 * kThreads;              // Theorem 3: at most four undecided rounds per query
+constexpr int kBatchRowBytes = 36;                     // staged row: 31 entries + pad; 9 words keep 32 rows on 32 banks
+
 __global__ void __launch_bounds__(kThreads)
 schedule_batch_kernel(const int32_t *__restrict__ p_in, const int32_t *__restrict__ rank_in,
                       const int32_t *__restrict__ root_in, int64_t nq, int row_stride,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
                       int32_t *bad_count, int recv_vec_ok, int send_vec_ok)
 {
-    // rows are staged 31 bytes wide and padded while they are written out
-    __shared__ uint32_t stage[kWarpsPerBlock][2][kMaxRowBytes * 32 / 4];
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int64_t n_tiles = (nq + 31) >> 5;
-    const int64_t warps_total = (int64_t)gridDim.x * kWarpsPerBlock;
-    const ByteRow recv_row{reinterpret_cast<int8_t *>(stage[warp][0]) + lane * kMaxRowBytes};
-    const ByteRow send_row{reinterpret_cast<int8_t *>(stage[warp][1]) + lane * kMaxRowBytes};
+    __shared__ uint32_t stage[2][kThreads * kBatchRowBytes / 4];
+    __shared__ uint32_t query_p[kThreads];             // p of the query in each row (0: nothing to compute)
+    __shared__ uint32_t query_r[kThreads];             // its virtual rank
+    __shared__ uint16_t order[kThreads];               // rows sorted by q, longest first
+    __shared__ int bin_count[32];
+    __shared__ int bin_start[32];
+    __shared__ uint16_t items[kBatchItems];            // undecided send entries: row | k << 8
+    __shared__ int n_items;
     const bool want_recv = recv_out != nullptr;
     const bool want_send = send_out != nullptr;
     constexpr int8_t kPadMark = -128;                  // no schedule entry is below -31
+    const int64_t n_tiles = (nq + kThreads - 1) / kThreads;
 
-    for (int64_t tile = (int64_t)blockIdx.x * kWarpsPerBlock + warp; tile < n_tiles; tile += warps_total) {
-        const int64_t first = tile << 5;
-        const int64_t idx = first + lane;
-        if (idx < nq) {
-            const int32_t pi = p_in[idx], ai = rank_in[idx], ri = root_in[idx];
-            int q = 0;
-            const bool ok = pi >= 1 && ai >= 0 && ai < pi && ri >= 0 && ri < pi;
-            if (!ok) {
-                if (bad_count) atomicAdd(bad_count, 1);
-            } else if (pi >= 2) {
-                const Geometry g = make_geometry((uint32_t)pi);
-                q = g.q;
-                const uint32_t a = (uint32_t)ai, root = (uint32_t)ri;
-                const uint32_t r = a >= root ? a - root : a + ((uint32_t)pi - root);
-                NoStats ns;
-                rank_rows(g, r, recv_row, send_row, want_recv, want_send, ns);
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int64_t first = tile * kThreads;
+        const int rows = (int)min((int64_t)kThreads, nq - first);
+        if (threadIdx.x < 32) bin_count[threadIdx.x] = 0;
+        if (threadIdx.x == 32) n_items = 0;
+        __syncthreads();                               // previous tile flushed, bins cleared
+        int q = 0, slot = 0;
+        {
+            uint32_t p = 0, r = 0;
+            if ((int)threadIdx.x < rows) {
+                const int64_t idx = first + threadIdx.x;
+                const int32_t pi = p_in[idx], ai = rank_in[idx], ri = root_in[idx];
+                const bool ok = pi >= 1 && ai >= 0 && ai < pi && ri >= 0 && ri < pi;
+                if (!ok) {
+                    if (bad_count) atomicAdd(bad_count, 1);
+                } else if (pi >= 2) {
+                    p = (uint32_t)pi;
+                    q = 32 - __clz(p - 1u);
+                    r = ai >= ri ? (uint32_t)(ai - ri) : (uint32_t)ai + (p - (uint32_t)ri);
+                }
             }
-            for (int k = q; k < kMaxRowBytes; ++k) { recv_row(k, kPadMark); send_row(k, kPadMark); }
+            query_p[threadIdx.x] = p;
+            query_r[threadIdx.x] = r;
+            slot = atomicAdd(&bin_count[q], 1);
         }
-        __syncwarp();
-        const int rows = (int)min((int64_t)32, nq - first);
+        __syncthreads();
+        if (threadIdx.x < 32) {                        // bins in descending q: start = rows with a larger q
+            int above = 0;
+            for (int b = threadIdx.x + 1; b < 32; ++b) above += bin_count[b];
+            bin_start[threadIdx.x] = above;
+        }
+        __syncthreads();
+        order[bin_start[q] + slot] = (uint16_t)threadIdx.x;
+        __syncthreads();
+
+        {
+            const int row = order[threadIdx.x];
+            const uint32_t p = query_p[row];
+            const ByteRow recv_row{reinterpret_cast<int8_t *>(stage[0]) + row * kBatchRowBytes};
+            const ByteRow send_row{reinterpret_cast<int8_t *>(stage[1]) + row * kBatchRowBytes};
+            int qq = 0;
+            uint32_t viol = 0;
+            if (p >= 2u) {
+                const Geometry g = make_geometry(p);
+                qq = g.q;
+                const uint32_t r = query_r[row];
+                NoStats ns;
+                const int b = want_recv ? recv_search_fast(g, r, qq - 1, recv_row, ns) : baseblock(g, r);
+                if (want_send) {
+                    if (r == 0u) {
+                        for (int k = 0; k < qq; ++k) send_row(k, k);
+                    } else {
+                        viol = send_walk(g, r, b, send_row);
+                    }
+                }
+            }
+            for (int k = qq; k < kMaxRowBytes; ++k) { recv_row(k, kPadMark); send_row(k, kPadMark); }
+            // Rounds Algorithm 6 could not decide (at most four per query, Theorem 3) are queued
+            // for the whole block, so that the lanes that have one do not hold up the others;
+            // a warp's items stay together, which keeps like q side by side.
+            const int lane = threadIdx.x & 31;
+            while (__any_sync(0xffffffffu, viol != 0u)) {
+                const bool has = viol != 0u;
+                const unsigned int mask = __ballot_sync(0xffffffffu, has);
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&n_items, __popc(mask));
+                base = __shfl_sync(0xffffffffu, base, 0);
+                if (has) {
+                    const int k = 31 - __clz(viol);
+                    viol ^= 1u << k;
+                    const int at = base + __popc(mask & ((1u << lane) - 1u));
+                    if (at < kBatchItems) {
+                        items[at] = (uint16_t)(row | (k << 8));
+                    } else {                               // cannot happen by Theorem 3; done on the spot
+                        const Geometry g = make_geometry(p);
+                        uint32_t t = query_r[row] + skip_of(g, k);
+                        if (t >= g.p) t -= g.p;
+                        NoStats ns;
+                        send_row(k, recv_entry(g, t, k, ns));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        {
+            const int n = min(n_items, kBatchItems);
+            for (int i = threadIdx.x; i < n; i += kThreads) {
+                const int row = items[i] & 255;
+                const int k = items[i] >> 8;
+                const Geometry g = make_geometry(query_p[row]);
+                uint32_t t = query_r[row] + skip_of(g, k);
+                if (t >= g.p) t -= g.p;
+                NoStats ns;
+                const ByteRow send_row{reinterpret_cast<int8_t *>(stage[1]) + row * kBatchRowBytes};
+                send_row(k, recv_entry(g, t, k, ns));      // Section 2.3: recvblock[k] of the to-processor
+            }
+        }
+        __syncthreads();
+
         const int n_entries = rows * row_stride;
         for (int t = 0; t < 2; ++t) {
             int32_t *out = t == 0 ? recv_out : send_out;
             if (out == nullptr) continue;
             out += (size_t)first * (size_t)row_stride;
-            const int8_t *bytes = reinterpret_cast<const int8_t *>(stage[warp][t]);
+            const int8_t *bytes = reinterpret_cast<const int8_t *>(stage[t]);
             const bool vec_ok = (t == 0 ? recv_vec_ok : send_vec_ok) && (row_stride & 3) == 0;
             if (vec_ok) {
                 int4 *out4 = reinterpret_cast<int4 *>(out);
                 const int nvec = n_entries >> 2;
                 const int vec_per_row = row_stride >> 2;
-                for (int i = lane; i < nvec; i += 32) {
+                for (int i = threadIdx.x; i < nvec; i += kThreads) {
                     const int row = i / vec_per_row;
                     const int col = (i - row * vec_per_row) << 2;
                     int e[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const int cc = col + j;
-                        const int val = cc < kMaxRowBytes ? (int)bytes[row * kMaxRowBytes + cc] : (int)kPadMark;
+                        const int val = cc < kMaxRowBytes ? (int)bytes[row * kBatchRowBytes + cc] : (int)kPadMark;
                         e[j] = val == (int)kPadMark ? BCAST_PAD : val;
                     }
                     __stcs(out4 + i, make_int4(e[0], e[1], e[2], e[3]));
                 }
             } else {
-                for (int i = lane; i < n_entries; i += 32) {
+                for (int i = threadIdx.x; i < n_entries; i += kThreads) {
                     const int row = i / row_stride;
                     const int cc = i - row * row_stride;
-                    const int val = cc < kMaxRowBytes ? (int)bytes[row * kMaxRowBytes + cc] : (int)kPadMark;
+                    const int val = cc < kMaxRowBytes ? (int)bytes[row * kBatchRowBytes + cc] : (int)kPadMark;
                     __stcs(out + i, val == (int)kPadMark ? BCAST_PAD : val);
                 }
             }
         }
-        __syncwarp();
     }
 }
 
@@ -914,10 +1002,9 @@ int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const in
     if (nq == 0) return BCAST_OK;
     const int sms = sm_count();
     if (sms <= 0) return BCAST_ECUDA;
-    const int64_t n_tiles = (nq + 31) / 32;
-    const int64_t blocks_needed = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    // one warp tile per warp while that keeps the grid below 2^20 blocks: short-lived blocks
-    // balance better than a resident grid striding over the tiles
+    const int64_t blocks_needed = (nq + kThreads - 1) / kThreads;
+    // one tile of kThreads queries per block while that keeps the grid below 2^20 blocks:
+    // short-lived blocks balance better than a resident grid striding over the tiles
     const int64_t grid_cap = (int64_t)1 << 20;
     const int grid = (int)(blocks_needed < grid_cap ? blocks_needed : grid_cap);
     schedule_batch_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
