@@ -303,4 +303,29 @@ int64_t bcast_round_block(int32_t q, int64_t n, int64_t j, const int32_t *sched_
 }
 #endif
 
+/*
+ * The same lookup as bcast_round_block for use inside the caller's own code,
+ * host or device (a kernel that moves the blocks reads its row from the table
+ * and calls this once per round): Theorem 1's block sched_row[k] + q*floor(i/q) - x
+ * with i = x + j, k = i mod q.  No argument checks: q >= 1, n >= 1,
+ * 0 <= j < n-1+q are the caller's duty.  *k_out (may be NULL) receives the skip
+ * index of the round.  Returns the block, capped to n-1, or BCAST_NONE.
+ */
+#if defined(__CUDACC__)
+#define BCAST_INLINE static __host__ __device__ __forceinline__
+#else
+#define BCAST_INLINE static inline
+#endif
+BCAST_INLINE int64_t bcast_round_block_inline(int32_t q, int64_t n, int64_t j, const int32_t *sched_row,
+                                              int32_t *k_out)
+{
+    const int64_t x = (q - (n - 1) % q) % q;
+    const int64_t i = x + j;
+    const int32_t k = (int32_t)(i % q);
+    const int64_t raw = (int64_t)sched_row[k] + (i / q) * q - x;
+    if (k_out) *k_out = k;
+    if (raw < 0) return BCAST_NONE;
+    return raw > n - 1 ? n - 1 : raw;
+}
+
 #endif /* BCAST_SCHED_H */

@@ -16,7 +16,8 @@ from conftest import ROOT
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "bcast_sched.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(bcast_[a-z_0-9]+)\s*\(", text)))
+    names = set(re.findall(r"\b(bcast_[a-z_0-9]+)\s*\(", text))
+    return sorted(n for n in names if not n.endswith("_inline"))      # inline helpers are not exported
 
 
 def test_library_exports_every_declared_symbol():
@@ -52,6 +53,30 @@ def test_round_lookup_matches_oracle():
                 assert bs.bcast_round_block(q, n, j, row) == oracle.round_block(q, n, j, row)
                 x = (q - (n - 1) % q) % q
                 assert shift == q * ((x + j) // q) - x
+
+
+def test_inline_round_lookup_compiles_as_c_and_matches_oracle(tmp_path):
+    # the header's inline form of the lookup, built with a plain C compiler
+    import subprocess
+    src = tmp_path / "shim.c"
+    src.write_text('#include "bcast_sched.h"\n'
+                   'long long shim(int q, long long n, long long j, const int *row, int *k)\n'
+                   '{ return bcast_round_block_inline(q, n, j, row, k); }\n')
+    lib_path = tmp_path / "shim.so"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-shared", "-fPIC", "-I", os.path.join(ROOT, "include"),
+                           "-o", str(lib_path), str(src)])
+    shim = ctypes.CDLL(str(lib_path)).shim
+    shim.restype = ctypes.c_longlong
+    shim.argtypes = [ctypes.c_int, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_void_p, ctypes.POINTER(ctypes.c_int)]
+    rng = np.random.default_rng(9)
+    for q in range(1, 12):
+        for n in list(range(1, 30)) + [1000]:
+            row = rng.integers(-q, q, q).astype(np.int32)
+            total = n - 1 + q
+            for j in (range(total) if total < 60 else [0, 1, q, total // 2, total - 1]):
+                k = ctypes.c_int(-1)
+                assert shim(q, n, j, row.ctypes.data, ctypes.byref(k)) == oracle.round_block(q, n, j, row)
+                assert k.value == oracle.round_k(q, n, j)
 
 
 def test_host_argument_errors():
