@@ -518,12 +518,12 @@ def build_other(args, torch, bs):
                                                              % (n, small_p))
 
     # contributions copied in (16 B per cell), sent counts cleared and read (2 B per cell), byte tables, and per
-    # round and processor: two table bytes, wire block and value written and read, one value read, one value
-    # read-modify-write, sent count read twice and written once
-    nbytes = p * (10 * q + 18 * n + rounds * (2 + 24 + 8 + 16 + 3))
+    # round and processor: three table bytes, the sender's value read, the own value read and written, sent
+    # count read twice and written once
+    nbytes = p * (10 * q + 18 * n + rounds * (3 + 8 + 16 + 3))
     return dict(label="Observation 1.3's reduction by all processors of p=%d (q=%d), n=%d blocks, %d rounds"
                       % (p, q, n, rounds), metric="simulated_partial_results_per_s", unit="blocks/s",
-                units=(p - 1) * n, bytes=nbytes, step=step, launches=2 * rounds + 4, kernel="reduce_recv_kernel",
+                units=(p - 1) * n, bytes=nbytes, step=step, launches=rounds + 4, kernel="reduce_round_kernel",
                 bound="hbm", e2e=e2e_step, h2d=0, d2h=64 + 8 * n, oracle=oracle_sample,
                 extra=lambda: {"stats": stats.tolist()})
 

@@ -275,7 +275,7 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
  *   [7] unused, 0
  * scratch_dev: at least bcast_simulate_scratch_bytes(p, n, 1) bytes, 16-byte
  * aligned.  Tables, limits, asynchrony and return value as for
- * bcast_simulate_broadcast; two launches per round.
+ * bcast_simulate_broadcast.
  */
 int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
                           const int32_t *recvblock_dev, const int32_t *sendblock_dev,

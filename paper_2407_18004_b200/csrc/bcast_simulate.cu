@@ -9,16 +9,15 @@
 //     processor from each table, consecutive processors from consecutive addresses, and the
 //     2q*P bytes stay in L2 over the n-1+q rounds.  Entries outside [-q, q-1] are counted
 //     and stored as kInvalid, which moves nothing in any round.
-//   * One thread per processor, one launch per round (two for the reduction: everybody
-//     sends, then everybody receives), all on the caller's stream.  Nothing waits on
-//     another block inside a launch.
+//   * One thread per processor, one launch per round, all on the caller's stream.  Nothing
+//     waits on another block inside a launch.
 //   * Broadcast state is arrival[b][a], the round in which processor a got block b.  A
 //     sender "held the block before the round" iff its arrival is in [0, round); a value
 //     written during the round is >= round, so concurrent readers decide the same way
 //     whether or not they see it: one buffer, no race in the outcome.
-//   * Reduction state is value[b][a] plus a saturating count sent[b][a]; the messages of a
-//     round go through wire arrays (block, value) written by the send launch and read by
-//     the receive launch.
+//   * Reduction state is value[b][a] plus a saturating count sent[b][a]; a receiver reads its
+//     to-processor's partial result in place (see reduce_round_kernel for why the outcome
+//     does not depend on the order of the threads).
 //   * Counters are summed per warp with redux, per block in shared memory, and added to the
 //     64-bit statistics with one atomic per block and counter that is not zero.
 #include <cuda_runtime.h>
@@ -167,66 +166,51 @@ count_missing_kernel(const int32_t *__restrict__ arrival, size_t cells, unsigned
 }
 
 // ------------------------------------------------------------------ reduction (reversed rounds)
-// First half of a reduction round: processor a puts its partial result of the block it
-// RECEIVED in the corresponding broadcast round on the wire (the root sends nothing).
+// One reduction round for every processor.  Processor a sends its partial result of the block
+// it RECEIVED in the corresponding broadcast round to its from-processor (the root sends
+// nothing), and takes, from its to-processor t, a partial result of the block it SENT to t in
+// that broadcast round, which it adds to its own; then it notes its own send as done.
+//
+// The receiver reads the sender's value in place, in the same launch, and the outcome does
+// not depend on the order of the threads: value[b][t] is read by t's from-processor only when
+// t sends b in this round, and t adds to value[b][t] only when it receives b and is NOT
+// sending b (a processor that receives the block it is sending would never pass the sum on,
+// which is counted instead); sent[.][a] is read and written by thread a alone.
 __global__ void __launch_bounds__(kThreads)
-reduce_send_kernel(const int8_t *__restrict__ recv_k, const uint64_t *__restrict__ value,
-                   const uint8_t *__restrict__ sent, int32_t *__restrict__ wire_block,
-                   uint64_t *__restrict__ wire_value, uint32_t p, uint32_t root, int64_t n,
-                   int64_t shift, unsigned long long *stats)
+reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
+                    uint64_t *value, uint8_t *sent, uint32_t p, uint32_t root, int64_t n,
+                    uint32_t skip_k, int64_t shift, unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
-    unsigned int c2 = 0;
-    if (a < p) {
-        const int64_t blk = a == root ? -1 : block_of(recv_k[a], shift, n);
-        wire_block[a] = (int32_t)blk;                      // n - 1 < 2^31 is checked on the host
-        if (blk >= 0) {
-            wire_value[a] = value[(size_t)blk * p + a];
-            if (sent[(size_t)blk * p + a] > 0) c2 = 1;
-        }
-    }
-    add_stat(bstats, 2, c2);
-    stats_end(bstats, stats);
-}
-
-// Second half: processor a takes, from its to-processor t, a partial result of the block it
-// SENT to t in the corresponding broadcast round and adds it to its own; then it notes its
-// own send of this round as done.
-__global__ void __launch_bounds__(kThreads)
-reduce_recv_kernel(const int8_t *__restrict__ send_k, uint64_t *value, uint8_t *sent,
-                   const int32_t *__restrict__ wire_block, const uint64_t *__restrict__ wire_value,
-                   uint32_t p, uint32_t root, int64_t n, uint32_t skip_k, int64_t shift,
-                   unsigned long long *stats)
-{
-    __shared__ BlockStats bstats;
-    stats_begin(bstats);
-    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
-    unsigned int c0 = 0, c1 = 0, c3 = 0, c6 = 0;
+    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
     if (a < p) {
         uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
         if (t >= p) t -= p;
+        const int64_t mine = a == root ? -1 : block_of(recv_k[a], shift, n);       // what a sends
+        const int64_t got = t == root ? -1 : block_of(recv_k[t], shift, n);        // what t sends to a
         const int64_t want = t == root ? -1 : block_of(send_k[a], shift, n);
-        const int64_t mine = wire_block[a];
-        const int64_t got = t == root ? -1 : (int64_t)wire_block[t];
+        uint8_t sent_mine = 0;
+        if (mine >= 0) {
+            sent_mine = sent[(size_t)mine * p + a];
+            if (sent_mine > 0) c2 = 1;
+        }
         if (want < 0) {
             if (got >= 0) c3 = 1;
         } else if (got != want) {
             c0 = 1;
-        } else if (a != root && (sent[(size_t)want * p + a] > 0 || mine == want)) {
+        } else if (a != root && (mine == want || sent[(size_t)want * p + a] > 0)) {
             c1 = 1;                                        // it would never be passed on
         } else {
-            value[(size_t)want * p + a] += wire_value[t];
+            value[(size_t)want * p + a] += value[(size_t)want * p + t];
             c6 = 1;
         }
-        if (mine >= 0) {
-            const uint8_t before = sent[(size_t)mine * p + a];
-            if (before < 2) sent[(size_t)mine * p + a] = before + 1;
-        }
+        if (mine >= 0 && sent_mine < 2) sent[(size_t)mine * p + a] = sent_mine + 1;
     }
     add_stat(bstats, 0, c0);
     add_stat(bstats, 1, c1);
+    add_stat(bstats, 2, c2);
     add_stat(bstats, 3, c3);
     add_stat(bstats, 6, c6);
     stats_end(bstats, stats);
@@ -302,7 +286,7 @@ int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction)
     const int q = host_q(p);
     const int64_t P = padded(p);
     int64_t bytes = kHeaderBytes + 2 * (int64_t)q * P;
-    if (reduction) bytes += 8 * P + 4 * P + n * (int64_t)p;        // wire values, wire blocks, sent counts
+    if (reduction) bytes += n * (int64_t)p;                        // sent counts
     return bytes;
 }
 
@@ -377,9 +361,7 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
     if (scratch_bytes < bcast_simulate_scratch_bytes(p, n, 1)) return BCAST_ESCRATCH;
     int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
     int8_t *send_t = recv_t + (size_t)q * plan.P;
-    uint64_t *wire_value = reinterpret_cast<uint64_t *>(send_t + (size_t)q * plan.P);
-    int32_t *wire_block = reinterpret_cast<int32_t *>(wire_value + plan.P);
-    uint8_t *sent = reinterpret_cast<uint8_t *>(wire_block + plan.P);
+    uint8_t *sent = reinterpret_cast<uint8_t *>(send_t + (size_t)q * plan.P);
     if (cudaMemsetAsync(sent, 0, (size_t)n * (size_t)p, stream) != cudaSuccess) return BCAST_ECUDA;
     const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
     transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
@@ -389,12 +371,9 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
         const int64_t i = plan.x + j;
         const int k = (int)(i % q);
         const int64_t shift = (i / q) * q - plan.x;
-        reduce_send_kernel<<<blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, value_dev, sent,
-                                                            wire_block, wire_value, (uint32_t)p, (uint32_t)root,
-                                                            n, shift, stats);
-        reduce_recv_kernel<<<blocks, kThreads, 0, stream>>>(send_t + (size_t)k * plan.P, value_dev, sent,
-                                                            wire_block, wire_value, (uint32_t)p, (uint32_t)root,
-                                                            n, plan.skip[k], shift, stats);
+        reduce_round_kernel<<<blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P,
+                                                             value_dev, sent, (uint32_t)p, (uint32_t)root, n,
+                                                             plan.skip[k], shift, stats);
     }
     for (int64_t b0 = 0; b0 < n; b0 += 65535) {
         const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
