@@ -80,6 +80,10 @@ int bcast_skips(int32_t p, int32_t *skip_host);
  * the vector-store path).  Either table pointer may be NULL to skip that table,
  * not both.  An empty rank range and p = 1 (q = 0) succeed without a launch.
  * Asynchronous on cuda_stream.  Returns q.
+ * The kernel has two launch shapes, chosen per call from an estimate of how
+ * many entries of this p need the search of Algorithms 4 and 5; the environment
+ * variable BCAST_LAUNCH_SHAPE=block|warps forces one (tuning, tests).  The
+ * tables are the same either way.
  */
 int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
                    int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);

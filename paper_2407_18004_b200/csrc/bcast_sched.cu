@@ -24,6 +24,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <stdlib.h>
+#include <string.h>
+
 #include <mutex>
 
 #include "../../include/bcast_sched.h"
@@ -179,15 +182,26 @@ struct SearchItem {
     uint16_t table;
 };
 
-constexpr int kSearchCapacity = 2 * kThreads;
-constexpr int kCopyCapacity = 2 * kThreads;
-
-struct TileQueue {
+// A queue serves a GROUP of consecutive rows of the tile whose threads drain it together:
+// the whole tile (kGroup = kThreads, the threads meet at block barriers) or one warp's 32
+// rows (kGroup = 32, the warp goes through pass, drain and flush on its own and meets no
+// other warp).  Items never leave their group: a copy's source row lies in it.
+template <int kGroup>
+struct GroupQueue {
+    static constexpr int kGroupSize = kGroup;
+    static constexpr int kSearchCapacity = 2 * kGroup;
+    static constexpr int kCopyCapacity = 2 * kGroup;
     SearchItem search[kSearchCapacity];
     uint32_t copy[kCopyCapacity];               // src | dst << 9 | k << 18
     int n_search;
     int n_copy;
+    __device__ __forceinline__ static void sync()
+    {
+        if constexpr (kGroup == 32) __syncwarp(); else __syncthreads();
+    }
 };
+typedef GroupQueue<kThreads> TileQueue;
+typedef GroupQueue<32> WarpQueue;
 
 // Run the search for one item and drop the wanted entries into `row`.
 template <class Row, class Stats>
@@ -199,12 +213,12 @@ __device__ __forceinline__ void resolve_item(const Geometry &g, const SearchItem
 }
 
 // Queue a search; when the queue is full the calling thread does it on the spot.
-template <class Tile, class Stats>
-__device__ __forceinline__ void push_search(const Geometry &g, TileQueue &queue, const SearchItem &it,
+template <class Queue, class Tile, class Stats>
+__device__ __forceinline__ void push_search(const Geometry &g, Queue &queue, const SearchItem &it,
                                             const Tile &tile, Stats &stats)
 {
     const int slot = atomicAdd(&queue.n_search, 1);
-    if (slot < kSearchCapacity) {
+    if (slot < Queue::kSearchCapacity) {
         queue.search[slot] = it;
     } else {
         resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
@@ -212,16 +226,17 @@ __device__ __forceinline__ void push_search(const Geometry &g, TileQueue &queue,
 }
 
 // A send entry Algorithm 6 could not decide: round k of the rank in row `index`, virtual
-// rank r.  Its to-processor is a row of this tile whose receive entry will be final after
-// the tile's searches (then a copy is queued), or a rank that needs a search of its own.
-template <class Tile, class Stats>
+// rank r.  Its to-processor is a row of the same group whose receive entry will be final
+// after the group's searches (then a copy is queued), or a rank that needs a search of its own.
+template <class Queue, class Tile, class Stats>
 __device__ __forceinline__ void push_send_violation(const Geometry &g, uint32_t skip_k, int k, uint32_t r,
                                                     uint32_t index, uint32_t rows, bool want_recv,
-                                                    TileQueue &queue, const Tile &tile, Stats &stats)
+                                                    Queue &queue, const Tile &tile, Stats &stats)
 {
-    if (want_recv && index + skip_k < rows) {
+    if (want_recv && index + skip_k < rows &&
+        (index + skip_k) / Queue::kGroupSize == index / Queue::kGroupSize) {
         const int slot = atomicAdd(&queue.n_copy, 1);
-        if (slot < kCopyCapacity) {
+        if (slot < Queue::kCopyCapacity) {
             queue.copy[slot] = (index + skip_k) | (index << 9) | ((uint32_t)k << 18);
             return;
         }
@@ -246,11 +261,11 @@ __device__ __forceinline__ bool tile_can_share(const Geometry &g, uint32_t r_fir
 // high-level entries from it and walks only the low levels; without one each rank walks
 // all levels, with rank 1 as a stand-in for the root and for rows that are not real.  What
 // the pass cannot decide is queued.  Returns Algorithm 6's violations of this thread's rank.
-template <int Q, class Tile, class Stats>
+template <int Q, class Tile, class Queue, class Stats>
 __device__ __forceinline__ uint32_t tile_pass(const LevelTables &tab, const Geometry &g,
                                               const TileRuns<typename WalkInt<Q>::type> &runs,
                                               uint32_t r_first, uint32_t rows, const Tile &tile,
-                                              bool want_recv, bool want_send, TileQueue &queue, Stats &stats)
+                                              bool want_recv, bool want_send, Queue &queue, Stats &stats)
 {
     const uint32_t index = threadIdx.x;
     const bool active = index < rows;
@@ -270,9 +285,11 @@ __device__ __forceinline__ uint32_t tile_pass(const LevelTables &tab, const Geom
             auto st = apply_tile_runs<Q>(runs, (int)index, recv_row, send_row);
             closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
             closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
-            // entries of the high levels that the description left undecided
-            if ((int)index < runs.n_pending) {
-                const uint32_t item = runs.pending[index];
+            // entries of the high levels that the description left undecided (at most kMaxPending = 32,
+            // so the threads of one group see them all); each goes to the queue of its row's group
+            const uint32_t member = index % Queue::kGroupSize;
+            const uint32_t item = (int)member < runs.n_pending ? runs.pending[member] : 0xffffffffu;
+            if (item != 0xffffffffu && (item & 511u) / Queue::kGroupSize == index / Queue::kGroupSize) {
                 const uint32_t row = item & 511u;
                 const int k = (int)((item >> 9) & 31u);
                 const uint32_t rr = r_first + row;
@@ -308,21 +325,23 @@ __device__ __forceinline__ uint32_t tile_pass(const LevelTables &tab, const Geom
     return send_flags;
 }
 
-// After the closed-form pass of a tile and a barrier: searches, then (after another
-// barrier, only if needed) the copies.  Every thread of the block calls this.
-template <class Tile, class Stats>
-__device__ __forceinline__ void drain_queue(const Geometry &g, TileQueue &queue, const Tile &tile, Stats &stats)
+// After the closed-form pass of a group's rows and its barrier: searches, then (after another
+// barrier, only if needed) the copies.  Every thread of the group calls this.
+template <class Queue, class Tile, class Stats>
+__device__ __forceinline__ void drain_queue(const Geometry &g, Queue &queue, const Tile &tile, Stats &stats)
 {
-    const int n_search = min(queue.n_search, kSearchCapacity);
-    const int n_copy = min(queue.n_copy, kCopyCapacity);
-    for (int i = threadIdx.x; i < n_search; i += kThreads) {
+    constexpr int kGroup = Queue::kGroupSize;
+    const int member = threadIdx.x % kGroup;
+    const int n_search = min(queue.n_search, Queue::kSearchCapacity);
+    const int n_copy = min(queue.n_copy, Queue::kCopyCapacity);
+    for (int i = member; i < n_search; i += kGroup) {
         const SearchItem it = queue.search[i];
         // one call site: items for either table run the same instructions side by side
         resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
     }
     if (n_copy > 0) {
-        __syncthreads();                                   // n_copy is the same for every thread
-        for (int i = threadIdx.x; i < n_copy; i += kThreads) {
+        Queue::sync();                                     // n_copy is the same for every thread of the group
+        for (int i = member; i < n_copy; i += kGroup) {
             const uint32_t c = queue.copy[i];
             const int k = (int)(c >> 18);
             tile.send_row((c >> 9) & 511u)(k, tile.recv_row(c & 511u).get(k));
@@ -345,16 +364,167 @@ struct SharedTile {
     __device__ __forceinline__ ByteRow send_row(uint32_t i) const { return ByteRow{send + slot(i) * Q}; }
 };
 
+// ------------------------------------------------------------------ warps on their own, searches deferred
+// The launch shape of bcast_schedule proper.  After the run descriptions are built no warp
+// waits for another: each takes its own 32 rows of every tile through the closed-form pass
+// and streams them out at once, undecided entries included (with whatever the pass left
+// there).  What is undecided goes to ONE queue per block, and when all tiles are out the
+// whole block runs the searches side by side, every lane busy, and stores each found entry
+// straight into the output table, over the placeholder.  (Per tile, the undecided entries of
+// 256 rows keep only a third of a block's lanes busy; per warp even fewer.)
+//
+// A deferred item names a virtual rank whose receive schedule is searched, the output row
+// (relative to the block's first row) and two sets of rounds:
+//   own rows  (kind 0): recv_mask  - rounds of the row's receive entries;
+//                       other_mask - rounds k whose value ALSO is the send entry of the row
+//                                    skip[k] above (its to-processor is this row, Section 2.3),
+//                                    noted by that row's lane when Algorithm 6 could not
+//                                    decide it and both rows belong to the same warp;
+//   send only (kind 1): other_mask - rounds k of the row's SEND entries, `rank` being the
+//                                    row's to-processor for that round.
+struct DeferredItem {
+    uint32_t rank;
+    uint32_t row_kind;                                     // row | kind << 31
+    uint32_t recv_mask;
+    uint32_t other_mask;
+};
+
+constexpr int kDeferredCapacity = 384;
+
+struct DeferredQueue {
+    DeferredItem items[kDeferredCapacity];
+    uint32_t need_recv[kWarpsPerBlock][32];                // per warp and row of its slice: rounds to search
+    uint32_t need_partner[kWarpsPerBlock][32];             // rounds whose value the row skip[k] above sends
+    int n;
+};
+
+union QueueStorage {
+    TileQueue tile;                                        // one queue for the block, or
+    DeferredQueue deferred;                                // the block's deferred searches
+};
+
+// Search for one deferred item; emit(table, row, k, value) receives every wanted entry
+// (table 0 = receive, 1 = send; row relative to the block's first row).
+template <class Emit>
+__device__ __forceinline__ void resolve_deferred(const Geometry &g, const LevelTables &tab, const DeferredItem &it,
+                                                 Emit emit)
+{
+    const uint32_t row = it.row_kind & 0x7fffffffu;
+    const bool send_only = (it.row_kind >> 31) != 0u;
+    const uint32_t recv_mask = it.recv_mask, other_mask = it.other_mask;
+    NoStats ns;
+    recv_search_fast(g, it.rank, 31 - __clz(recv_mask | other_mask), [&](int k, int val) {
+        if ((recv_mask >> k) & 1u) emit(0, row, k, val);
+        if ((other_mask >> k) & 1u) emit(1, send_only ? row : row - tab.skip[k], k, val);
+    }, ns);
+}
+
+// The closed-form pass of one warp's 32 rows of a tile (lane l owns row 32*warp + l).  Rounds
+// the pass cannot decide become deferred items; when the block's queue is full the lane runs
+// the search itself and puts the entries into the staged rows, which are not flushed yet.
+template <int Q, class Tile>
+__device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry &g,
+                                          const TileRuns<typename WalkInt<Q>::type> &runs,
+                                          uint32_t r_first, uint32_t rows, uint32_t block_row0, const Tile &tile,
+                                          bool want_recv, bool want_send, DeferredQueue &dq)
+{
+    const uint32_t index = threadIdx.x;
+    const uint32_t lane = index & 31u;
+    const uint32_t warp = index >> 5;
+    uint32_t *need_recv = dq.need_recv[warp];
+    uint32_t *need_partner = dq.need_partner[warp];
+    const bool active = index < rows;
+    uint32_t r = 1u;
+    if (active) {
+        r = r_first + index;
+        if (r >= g.p) r -= g.p;
+    }
+    auto recv_row = tile.recv_row(index);
+    auto send_row = tile.send_row(index);
+    need_recv[lane] = 0u;
+    need_partner[lane] = 0u;
+    __syncwarp();
+
+    auto defer = [&](const DeferredItem &it) {
+        const int slot = atomicAdd(&dq.n, 1);
+        if (slot < kDeferredCapacity) {
+            dq.items[slot] = it;
+        } else {
+            resolve_deferred(g, tab, it, [&](int table, uint32_t row, int k, int val) {
+                const uint32_t in_tile = row - block_row0;
+                if (table == 0) tile.recv_row(in_tile)(k, val); else tile.send_row(in_tile)(k, val);
+            });
+        }
+    };
+    // Algorithm 6 could not decide round k of the send row of tile row `row` (virtual rank rr)
+    auto violation = [&](uint32_t row, int k, uint32_t rr) {
+        const uint32_t skip_k = tab.skip[k];
+        if (want_recv && (row & 31u) + skip_k < 32u && row + skip_k < rows) {
+            atomicOr(&need_partner[(row & 31u) + skip_k], 1u << k);      // the to-processor's lane will search it
+        } else {
+            uint32_t t = rr + skip_k;
+            if (t >= g.p) t -= g.p;
+            defer(DeferredItem{t, (block_row0 + row) | 0x80000000u, 0u, 1u << k});
+        }
+    };
+
+    uint32_t recv_flags = 0, send_flags = 0;
+    bool shared = false;
+    if constexpr (Q >= kSharedFrom + 2) {
+        shared = runs.n_runs > 0;                          // the same for the whole block
+        if (shared) {
+            auto st = apply_tile_runs<Q>(runs, (int)index, recv_row, send_row);
+            closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
+            closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
+            // entries of the high levels that the description left undecided (at most 32, one per
+            // lane); each warp takes those of its own rows, once their placeholders are written
+            __syncwarp();
+            const uint32_t item = (int)lane < runs.n_pending ? runs.pending[lane] : 0xffffffffu;
+            if (item != 0xffffffffu && (item & 511u) >> 5 == warp) {
+                const uint32_t row = item & 511u;
+                const int k = (int)((item >> 9) & 31u);
+                if ((item >> 14) & 1u) {
+                    if (want_send) violation(row, k, r_first + row);
+                } else if (want_recv) {
+                    atomicOr(&need_recv[row & 31u], 1u << k);
+                }
+            }
+        }
+    }
+    if (!shared) {
+        const bool is_root = r == 0u;
+        int b = 0;
+        recv_flags = closed_form_rows<Q>(tab, g.p, is_root ? 1u : r, recv_row, send_row, &send_flags, &b);
+        if (is_root) {                                     // the root sends block k in round k
+            for (int k = 0; k < Q; ++k) send_row(k, k);
+            recv_flags = (2u << (Q - 1)) - 1u;             // and its receive row comes from the search
+            send_flags = 0u;
+        }
+        if (!active) { recv_flags = 0u; send_flags = 0u; }
+    }
+    if (want_recv && recv_flags != 0u) atomicOr(&need_recv[lane], recv_flags);
+    uint32_t todo = want_send ? send_flags : 0u;
+    while (todo != 0u) {
+        const int k = 31 - __clz(todo);
+        todo ^= 1u << k;
+        violation(index, k, r);
+    }
+    __syncwarp();
+    const uint32_t mine = need_recv[lane], partner = need_partner[lane];
+    if ((mine | partner) != 0u) defer(DeferredItem{r, block_row0 + index, mine, partner});
+}
+
+
 template <int Q>
 __global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
 schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t anchor,
                       uint32_t row_begin, uint32_t n_ranks, int descending, int tiles_per_block,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
-                      int recv_vec_ok, int send_vec_ok, int shift_x)
+                      int recv_vec_ok, int send_vec_ok, int shift_x, int warps_alone)
 {
     typedef typename WalkInt<Q>::type Int;
     __shared__ uint32_t stage[2][(kThreads * Q + 15) / 16 * 4];   // byte tiles, kThreads rows of Q entries
-    __shared__ TileQueue queue;
+    __shared__ QueueStorage queues;
     __shared__ LevelTables lookup;                         // the tables again, for per-lane indices
     __shared__ TileRuns<Int> runs[kWarpsPerBlock];         // descriptions of the next kWarpsPerBlock tiles
     __shared__ uint32_t shift_words[32];                   // used only when shift_x != 0
@@ -399,6 +569,41 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         }
         if (!share && lane == 0) { runs[warp].n_runs = 0; runs[warp].n_pending = 0; }
     }
+    if (warps_alone) {                                     // host: only with ascending rows and no shift
+        DeferredQueue &dq = queues.deferred;
+        if (threadIdx.x == 0) dq.n = 0;
+        __syncthreads();                                   // descriptions built, queue empty
+        for (int slot = 0; slot < tiles_per_block; ++slot) {
+            const uint32_t t = group + (uint32_t)slot;
+            if (t >= n_tiles) break;
+            const uint32_t first = t * kThreads;
+            const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
+            const SharedTile<Q> tile{recv_bytes, send_bytes, rows, false};
+            warp_pass<Q>(tab, g, runs[slot], first_rank_of(first, rows), rows, (uint32_t)slot * kThreads, tile,
+                         want_recv, want_send, dq);
+            __syncwarp();                                  // the slice is staged
+            const uint32_t my_first = (uint32_t)warp * 32u;
+            if (my_first < rows) {
+                const int my_entries = (int)min(32u, rows - my_first) * Q;
+                const size_t base = (size_t)(first + my_first) * (size_t)Q;
+                const uint32_t word = my_first * Q / 4u;   // 32 rows of Q bytes are whole words
+                if (want_recv) flush_tile<32>(stage[0] + word, recv_out + base, my_entries, recv_vec_ok, lane);
+                if (want_send) flush_tile<32>(stage[1] + word, send_out + base, my_entries, send_vec_ok, lane);
+            }
+            __syncwarp();                                  // flushed before the next tile's pass overwrites it
+        }
+        __syncthreads();                                   // every slice is out; now the searches
+        const int n_deferred = min(dq.n, kDeferredCapacity);
+        const size_t block_base = (size_t)group * kThreads * (size_t)Q;
+        for (int i = threadIdx.x; i < n_deferred; i += kThreads) {
+            resolve_deferred(g, tab, dq.items[i], [&](int table, uint32_t row, int k, int val) {
+                int32_t *out = table == 0 ? recv_out : send_out;
+                out[block_base + (size_t)row * Q + k] = val;
+            });
+        }
+        return;
+    }
+    TileQueue &queue = queues.tile;
     for (int slot = 0; slot < tiles_per_block; ++slot) {
         const uint32_t t = group + (uint32_t)slot;
         if (t >= n_tiles) break;
@@ -872,6 +1077,53 @@ int bcast_skips(int32_t p, int32_t *skip_host)
     return q;
 }
 
+// Algorithm 6's violations of virtual rank r (1 <= r < p), counted on the host.
+static int host_violations(const LevelTables &tab, int64_t p, int q, int64_t r)
+{
+    int64_t rp = r, e = p;
+    int b = q;                                             // baseblock: only "b > 0" matters below
+    {
+        int64_t rem = r;
+        for (int k = q - 1; k >= 0; --k) {
+            if ((int64_t)tab.skip[k] == rem) { b = k; break; }
+            if ((int64_t)tab.skip[k] < rem) rem -= tab.skip[k];
+        }
+    }
+    int count = 0;
+    for (int k = q - 1; k >= 1; --k) {
+        const int64_t sk = tab.skip[k], sk_below = tab.skip[k - 1];
+        if (rp < sk) {
+            if (!(rp + sk < e || e < sk_below || (k == 1 && b > 0))) ++count;
+            if (e > sk) e = sk;
+        } else {
+            if (!(k == 1 || rp > sk || e - sk < sk_below) && rp + sk > e) ++count;
+            rp -= sk;
+            e -= sk;
+        }
+    }
+    return count;
+}
+
+// Which launch shape suits p: with few undecided entries per tile the warps go through the
+// tiles on their own and the block runs the few searches at the end (the deferred queue of a
+// block holds kDeferredCapacity items for up to kWarpsPerBlock tiles); with many, the block
+// meets after every tile and drains them there.  The density is estimated from Algorithm 6's
+// violations on a fixed sample of ranks; a wrong guess costs time, never correctness.
+static bool few_undecided_entries(const LevelTables &tab, int64_t p, int q)
+{
+    if (q < 2) return true;
+    const int kSamples = 80;
+    const int kMost = kSamples / 20;                       // at most 0.05 per rank
+    int total = 0;
+    uint64_t state = 0x9e3779b97f4a7c15ull ^ (uint64_t)p;
+    for (int i = 0; i < kSamples && total <= kMost; ++i) {
+        state = state * 6364136223846793005ull + 1442695040888963407ull;
+        const int64_t r = 1 + (int64_t)((state >> 33) % (uint64_t)(p - 1));
+        total += host_violations(tab, p, q, r);
+    }
+    return total <= kMost;
+}
+
 // Launch of the table kernel for n_rows output rows starting at global row index row_begin.
 static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int64_t n_rows, int descending,
                         int32_t *recv_dev, int32_t *send_dev, void *cuda_stream, int shift_x = 0)
@@ -884,16 +1136,30 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     int64_t tiles_per_block = n_tiles / ((int64_t)sms * kBlocksPerSmWanted);
     if (tiles_per_block < 1) tiles_per_block = 1;
     if (tiles_per_block > kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
+    if (const char *forced_tiles = getenv("BCAST_TILES_PER_BLOCK")) {          // tuning knob, 1..kWarpsPerBlock
+        const int v = atoi(forced_tiles);
+        if (v >= 1 && v <= kWarpsPerBlock) tiles_per_block = v;
+    }
     const int grid = (int)((n_tiles + tiles_per_block - 1) / tiles_per_block);
     const LevelTables tab = host_tables(p, q);
     const int recv_vec = ((uintptr_t)recv_dev & 15u) == 0, send_vec = ((uintptr_t)send_dev & 15u) == 0;
+    // BCAST_LAUNCH_SHAPE=block|warps overrides the estimate (for tuning and for the tests, which
+    // run both shapes on the same p); results never depend on it
+    bool few = false;
+    if (!descending && shift_x == 0) {
+        const char *forced = getenv("BCAST_LAUNCH_SHAPE");
+        if (forced != nullptr && strcmp(forced, "block") == 0) few = false;
+        else if (forced != nullptr && strcmp(forced, "warps") == 0) few = true;
+        else few = few_undecided_entries(tab, p, q);
+    }
+    const int warps_alone = few ? 1 : 0;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     switch (q) {
 #define BCAST_CASE(N)                                                                                     \
     case N:                                                                                               \
         schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)anchor,       \
             (uint32_t)row_begin, (uint32_t)n_rows, descending, (int)tiles_per_block, recv_dev, send_dev,  \
-            recv_vec, send_vec, shift_x);                                                                 \
+            recv_vec, send_vec, shift_x, warps_alone);                                                    \
         break;
         BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6) BCAST_CASE(7)
         BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12) BCAST_CASE(13)

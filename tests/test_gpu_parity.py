@@ -378,3 +378,24 @@ def test_table_kernel_against_batch_kernel_at_scale(p, root):
     assert int(bad) == 0
     assert bool((recv == brecv[:, :q]).all()), "receive tables differ"
     assert bool((send == bsend[:, :q]).all()), "send tables differ"
+
+
+# ------------------------------------------------------------------ both launch shapes of the table kernel
+@pytest.mark.parametrize("shape", ["block", "warps"])
+@pytest.mark.parametrize("p,root", [(1000, 0), (5000, 1234), (2 ** 16 + 1, 7), (300007, 299999), (2 ** 20 + 1, 0),
+                                    (2 ** 20 - 1, 5)])
+def test_both_launch_shapes_full_tables(monkeypatch, shape, p, root):
+    """The library picks the launch shape from an estimate; forced either way, on p with many and with few
+    undecided entries (the block's deferred queue overflows at p = 2^20 + 1), the tables equal the oracle's."""
+    monkeypatch.setenv("BCAST_LAUNCH_SHAPE", shape)
+    recv, send = gpu_tables(p, root)
+    orecv, osend = oracle.schedule_table(p, root)
+    assert_equal("recvblock (%s)" % shape, recv, orecv)
+    assert_equal("sendblock (%s)" % shape, send, osend)
+    # a ragged window that starts inside a warp's slice, and single tables
+    lo, hi = 37, min(p, 37 + 3 * 256 + 5)
+    r2, _ = bs.schedule(p, root, lo, hi, want_send=False)
+    _, s2 = bs.schedule(p, root, lo, hi, want_recv=False)
+    torch.cuda.synchronize()
+    assert_equal("recv window (%s)" % shape, r2.cpu().numpy(), orecv[lo:hi])
+    assert_equal("send window (%s)" % shape, s2.cpu().numpy(), osend[lo:hi])
