@@ -38,7 +38,7 @@ namespace bcast {
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 constexpr int kTableBlocksPerSm = 8;                   // resident blocks the table kernel is sized for
-constexpr int kSweepBlocksPerSm = 4;                   // resident blocks of the verification sweep
+constexpr int kSweepBlocksPerSm = 6;                   // resident blocks of the verification sweep
 constexpr int kBlocksPerSmWanted = 64;                 // grid size below which blocks take fewer tiles
 constexpr int kMaxRowBytes = 32;                       // staged row: q <= 31 bytes (+ pad in batch form)
 
