@@ -29,3 +29,18 @@ def test_reference_arm_single_process():
     assert out.returncode == 0, out.stderr[-2000:]
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["metric"] == "schedule_ranks_per_s"
+
+
+def test_reference_arm_other_modes():
+    # the oracle's leg of the other workloads, each on a small case
+    for args, metric in [(["--mode", "shifted", "--workload", "p=1000", "--blocks", "8"], "schedule_ranks_per_s"),
+                         (["--mode", "simulate", "--workload", "p=1000", "--blocks", "8"], "simulated_block_deliveries_per_s"),
+                         (["--mode", "reduce", "--workload", "p=1000", "--blocks", "8"], "simulated_partial_results_per_s"),
+                         (["--mode", "sweep", "--sweep-hi", "300"], "verified_rank_schedules_per_s"),
+                         (["--mode", "batch"], "schedule_queries_per_s")]:
+        out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                              "--warmup", "0"] + args, capture_output=True, text=True, timeout=300, cwd=ROOT)
+        assert out.returncode == 0, out.stderr[-2000:]
+        line = json.loads(out.stdout.strip().splitlines()[-1])
+        assert line["impl"] == "reference" and line["metric"] == metric and line["value"] > 0
+        assert line["cpu_baseline"]["kind"] == "oracle" and line["gpu_launches"] == 0
