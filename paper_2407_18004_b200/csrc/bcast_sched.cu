@@ -390,6 +390,7 @@ struct DeferredItem {
 };
 
 constexpr int kDeferredCapacity = 384;
+constexpr int kDescWarpsFromQ = 16;                    // smallest q with a descending-rows kernel of that shape
 
 struct DeferredQueue {
     DeferredItem items[kDeferredCapacity];
@@ -405,7 +406,7 @@ union QueueStorage {
 
 // Search for one deferred item; emit(table, row, k, value) receives every wanted entry
 // (table 0 = receive, 1 = send; row relative to the block's first row).
-template <class Emit>
+template <bool desc, class Emit>
 __device__ __forceinline__ void resolve_deferred(const Geometry &g, const LevelTables &tab, const DeferredItem &it,
                                                  Emit emit)
 {
@@ -415,28 +416,35 @@ __device__ __forceinline__ void resolve_deferred(const Geometry &g, const LevelT
     NoStats ns;
     recv_search_fast(g, it.rank, 31 - __clz(recv_mask | other_mask), [&](int k, int val) {
         if ((recv_mask >> k) & 1u) emit(0, row, k, val);
-        if ((other_mask >> k) & 1u) emit(1, send_only ? row : row - tab.skip[k], k, val);
+        // the row whose to-processor this row is: skip[k] ranks below, i.e. skip[k] rows above it when the
+        // rows are listed by descending rank
+        if ((other_mask >> k) & 1u)
+            emit(1, send_only ? row : (desc ? row + tab.skip[k] : row - tab.skip[k]), k, val);
     }, ns);
 }
 
 // The closed-form pass of one warp's 32 rows of a tile (lane l owns row 32*warp + l).  Rounds
 // the pass cannot decide become deferred items; when the block's queue is full the lane runs
 // the search itself and puts the entries into the staged rows, which are not flushed yet.
-template <int Q, class Tile>
+template <int Q, bool desc, class Tile>
 __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry &g,
                                           const TileRuns<typename WalkInt<Q>::type> &runs,
                                           uint32_t r_first, uint32_t rows, uint32_t block_row0, const Tile &tile,
                                           bool want_recv, bool want_send, DeferredQueue &dq)
 {
+    // index: the thread's row of the staged tile = its output row within the tile.  The ranks of a tile
+    // ascend with the row, or descend (Algorithm 7's tables); `ahead` is the thread's place counted from
+    // the tile's lowest rank r_first, which is how the run descriptions number the rows.
     const uint32_t index = threadIdx.x;
     const uint32_t lane = index & 31u;
     const uint32_t warp = index >> 5;
     uint32_t *need_recv = dq.need_recv[warp];
     uint32_t *need_partner = dq.need_partner[warp];
     const bool active = index < rows;
+    const uint32_t ahead = desc && active ? rows - 1u - index : index;
     uint32_t r = 1u;
     if (active) {
-        r = r_first + index;
+        r = r_first + ahead;
         if (r >= g.p) r -= g.p;
     }
     auto recv_row = tile.recv_row(index);
@@ -450,7 +458,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
         if (slot < kDeferredCapacity) {
             dq.items[slot] = it;
         } else {
-            resolve_deferred(g, tab, it, [&](int table, uint32_t row, int k, int val) {
+            resolve_deferred<desc>(g, tab, it, [&](int table, uint32_t row, int k, int val) {
                 const uint32_t in_tile = row - block_row0;
                 if (table == 0) tile.recv_row(in_tile)(k, val); else tile.send_row(in_tile)(k, val);
             });
@@ -459,8 +467,10 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     // Algorithm 6 could not decide round k of the send row of tile row `row` (virtual rank rr)
     auto violation = [&](uint32_t row, int k, uint32_t rr) {
         const uint32_t skip_k = tab.skip[k];
-        if (want_recv && (row & 31u) + skip_k < 32u && row + skip_k < rows) {
-            atomicOr(&need_partner[(row & 31u) + skip_k], 1u << k);      // the to-processor's lane will search it
+        // the to-processor's row: skip[k] ranks ahead; its lane will search the entry if it is in this warp
+        const bool near = desc ? (row & 31u) >= skip_k : (row & 31u) + skip_k < 32u && row + skip_k < rows;
+        if (want_recv && near) {
+            atomicOr(&need_partner[desc ? (row & 31u) - skip_k : (row & 31u) + skip_k], 1u << k);
         } else {
             uint32_t t = rr + skip_k;
             if (t >= g.p) t -= g.p;
@@ -473,18 +483,20 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     if constexpr (Q >= kSharedFrom + 2) {
         shared = runs.n_runs > 0;                          // the same for the whole block
         if (shared) {
-            auto st = apply_tile_runs<Q>(runs, (int)index, recv_row, send_row);
+            auto st = apply_tile_runs<Q>(runs, (int)ahead, recv_row, send_row);
             closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
             closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
             // entries of the high levels that the description left undecided (at most 32, one per
             // lane); each warp takes those of its own rows, once their placeholders are written
             __syncwarp();
             const uint32_t item = (int)lane < runs.n_pending ? runs.pending[lane] : 0xffffffffu;
-            if (item != 0xffffffffu && (item & 511u) >> 5 == warp) {
-                const uint32_t row = item & 511u;
+            // (a described tile is full, so place `a` from the lowest rank is row a, or row 255 - a)
+            const uint32_t item_row = desc ? (uint32_t)kThreads - 1u - (item & 511u) : (item & 511u);
+            if (item != 0xffffffffu && item_row >> 5 == warp) {
+                const uint32_t row = item_row;
                 const int k = (int)((item >> 9) & 31u);
                 if ((item >> 14) & 1u) {
-                    if (want_send) violation(row, k, r_first + row);
+                    if (want_send) violation(row, k, r_first + (item & 511u));
                 } else if (want_recv) {
                     atomicOr(&need_recv[row & 31u], 1u << k);
                 }
@@ -515,7 +527,11 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
 }
 
 
-template <int Q>
+// kDescWarps = false: the kernel of bcast_schedule and its variants, either launch shape, rows by
+// ascending rank in the warps-on-their-own shape.  kDescWarps = true: only that shape, rows by
+// descending rank (Algorithm 7's tables); a kernel of its own so that the other one is compiled
+// exactly as it would be without it.
+template <int Q, bool kDescWarps>
 __global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
 schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t anchor,
                       uint32_t row_begin, uint32_t n_ranks, int descending, int tiles_per_block,
@@ -569,7 +585,8 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         }
         if (!share && lane == 0) { runs[warp].n_runs = 0; runs[warp].n_pending = 0; }
     }
-    if (warps_alone) {                                     // host: only with ascending rows and no shift
+    if (kDescWarps || warps_alone) {                       // host: never with the shifted rows
+        constexpr bool desc = kDescWarps;
         DeferredQueue &dq = queues.deferred;
         if (threadIdx.x == 0) dq.n = 0;
         __syncthreads();                                   // descriptions built, queue empty
@@ -579,8 +596,8 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             const uint32_t first = t * kThreads;
             const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
             const SharedTile<Q> tile{recv_bytes, send_bytes, rows, false};
-            warp_pass<Q>(tab, g, runs[slot], first_rank_of(first, rows), rows, (uint32_t)slot * kThreads, tile,
-                         want_recv, want_send, dq);
+            warp_pass<Q, desc>(tab, g, runs[slot], first_rank_of(first, rows), rows, (uint32_t)slot * kThreads,
+                               tile, want_recv, want_send, dq);
             __syncwarp();                                  // the slice is staged
             const uint32_t my_first = (uint32_t)warp * 32u;
             if (my_first < rows) {
@@ -596,7 +613,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         const int n_deferred = min(dq.n, kDeferredCapacity);
         const size_t block_base = (size_t)group * kThreads * (size_t)Q;
         for (int i = threadIdx.x; i < n_deferred; i += kThreads) {
-            resolve_deferred(g, tab, dq.items[i], [&](int table, uint32_t row, int k, int val) {
+            resolve_deferred<desc>(g, tab, dq.items[i], [&](int table, uint32_t row, int k, int val) {
                 int32_t *out = table == 0 ? recv_out : send_out;
                 out[block_base + (size_t)row * Q + k] = val;
             });
@@ -1032,6 +1049,34 @@ static int64_t sweep_bytes_per_block(int32_t p_hi)
 
 constexpr int64_t kSweepHeaderBytes = 256;             // the work-queue counter lives here
 
+// Arguments of one launch of the table kernel, and the launch for a given q.
+struct TableLaunch {
+    LevelTables tab;
+    uint32_t p, anchor, row_begin, n_rows;
+    int descending, tiles_per_block;
+    int32_t *recv_dev, *send_dev;
+    int recv_vec, send_vec, shift_x, asc_warps;
+    bool desc_warps;
+    int grid;
+    cudaStream_t stream;
+};
+
+template <int N>
+static void launch_table_kernel(const TableLaunch &l)
+{
+    if constexpr (N >= kDescWarpsFromQ) {
+        if (l.desc_warps) {
+            schedule_table_kernel<N, true><<<l.grid, kThreads, 0, l.stream>>>(
+                l.tab, l.p, l.anchor, l.row_begin, l.n_rows, l.descending, l.tiles_per_block, l.recv_dev,
+                l.send_dev, l.recv_vec, l.send_vec, l.shift_x, 0);
+            return;
+        }
+    }
+    schedule_table_kernel<N, false><<<l.grid, kThreads, 0, l.stream>>>(
+        l.tab, l.p, l.anchor, l.row_begin, l.n_rows, l.descending, l.tiles_per_block, l.recv_dev, l.send_dev,
+        l.recv_vec, l.send_vec, l.shift_x, l.asc_warps);
+}
+
 }  // namespace bcast
 
 using namespace bcast;
@@ -1146,21 +1191,34 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     // BCAST_LAUNCH_SHAPE=block|warps overrides the estimate (for tuning and for the tests, which
     // run both shapes on the same p); results never depend on it
     bool few = false;
-    if (!descending && shift_x == 0) {
+    if (shift_x == 0) {
         const char *forced = getenv("BCAST_LAUNCH_SHAPE");
         if (forced != nullptr && strcmp(forced, "block") == 0) few = false;
         else if (forced != nullptr && strcmp(forced, "warps") == 0) few = true;
         else few = few_undecided_entries(tab, p, q);
     }
     const int warps_alone = few ? 1 : 0;
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // rows by descending rank take the warps-on-their-own shape only for q >= kDescWarpsFromQ (the
+    // sizes where it matters; each q is a kernel to compile), else the block-per-tile shape
+    TableLaunch launch;
+    launch.tab = tab;
+    launch.p = (uint32_t)p;
+    launch.anchor = (uint32_t)anchor;
+    launch.row_begin = (uint32_t)row_begin;
+    launch.n_rows = (uint32_t)n_rows;
+    launch.descending = descending;
+    launch.tiles_per_block = (int)tiles_per_block;
+    launch.recv_dev = recv_dev;
+    launch.send_dev = send_dev;
+    launch.recv_vec = recv_vec;
+    launch.send_vec = send_vec;
+    launch.shift_x = shift_x;
+    launch.asc_warps = !descending && warps_alone;
+    launch.desc_warps = descending && warps_alone && q >= kDescWarpsFromQ;
+    launch.grid = grid;
+    launch.stream = (cudaStream_t)cuda_stream;
     switch (q) {
-#define BCAST_CASE(N)                                                                                     \
-    case N:                                                                                               \
-        schedule_table_kernel<N><<<grid, kThreads, 0, stream>>>(tab, (uint32_t)p, (uint32_t)anchor,       \
-            (uint32_t)row_begin, (uint32_t)n_rows, descending, (int)tiles_per_block, recv_dev, send_dev,  \
-            recv_vec, send_vec, shift_x, warps_alone);                                                    \
-        break;
+#define BCAST_CASE(N) case N: launch_table_kernel<N>(launch); break;
         BCAST_CASE(1) BCAST_CASE(2) BCAST_CASE(3) BCAST_CASE(4) BCAST_CASE(5) BCAST_CASE(6) BCAST_CASE(7)
         BCAST_CASE(8) BCAST_CASE(9) BCAST_CASE(10) BCAST_CASE(11) BCAST_CASE(12) BCAST_CASE(13)
         BCAST_CASE(14) BCAST_CASE(15) BCAST_CASE(16) BCAST_CASE(17) BCAST_CASE(18) BCAST_CASE(19)

@@ -1,5 +1,7 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle,
 bit for bit, on the same seeded inputs."""
+import os
+
 import numpy as np
 import pytest
 
@@ -276,8 +278,11 @@ def test_schedule_host_chunks():
 
 # ------------------------------------------------------------------ Algorithm 7: all-broadcast tables
 @pytest.mark.parametrize("p,rank", [(2, 1), (17, 5), (1000, 0), (1000, 999), (1000, 417), (5000, 1234),
-                                    (70001, 69999), (2 ** 16 + 1, 3)])
-def test_allbroadcast_tables(p, rank):
+                                    (70001, 69999), (2 ** 16 + 1, 3), (2 ** 17 - 1, 77)])
+@pytest.mark.parametrize("shape", ["auto", "block", "warps"])
+def test_allbroadcast_tables(monkeypatch, shape, p, rank):
+    if shape != "auto":
+        monkeypatch.setenv("BCAST_LAUNCH_SHAPE", shape)        # both launch shapes of the table kernel
     orecv, osend = oracle.allbroadcast_schedule(p, rank)
     recv, send = bs.allbroadcast_schedule(p, rank)
     torch.cuda.synchronize()
@@ -295,6 +300,12 @@ def test_allbroadcast_large_p_is_the_reversed_broadcast_table():
     p, rank = workloads.P_MEDIUM, 777777
     recv0, send0 = bs.schedule(p)
     recv, send = bs.allbroadcast_schedule(p, rank)
+    os.environ["BCAST_LAUNCH_SHAPE"] = "warps"             # the other shape too (its deferred queue overflows here)
+    try:
+        recv_w, send_w = bs.allbroadcast_schedule(p, rank)
+    finally:
+        del os.environ["BCAST_LAUNCH_SHAPE"]
+    assert bool((recv_w == recv).all()) and bool((send_w == send).all())
     torch.cuda.synchronize()
     idx = (rank - torch.arange(p, device="cuda")) % p
     assert bool((recv == recv0[idx]).all()) and bool((send == send0[idx]).all())
