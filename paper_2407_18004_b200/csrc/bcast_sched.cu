@@ -1181,10 +1181,6 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     int64_t tiles_per_block = n_tiles / ((int64_t)sms * kBlocksPerSmWanted);
     if (tiles_per_block < 1) tiles_per_block = 1;
     if (tiles_per_block > kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
-    if (const char *forced_tiles = getenv("BCAST_TILES_PER_BLOCK")) {          // tuning knob, 1..kWarpsPerBlock
-        const int v = atoi(forced_tiles);
-        if (v >= 1 && v <= kWarpsPerBlock) tiles_per_block = v;
-    }
     const int grid = (int)((n_tiles + tiles_per_block - 1) / tiles_per_block);
     const LevelTables tab = host_tables(p, q);
     const int recv_vec = ((uintptr_t)recv_dev & 15u) == 0, send_vec = ((uintptr_t)send_dev & 15u) == 0;
