@@ -222,3 +222,16 @@ def test_shifted_tables_ranges_and_unaligned():
     with pytest.raises(bs.BcastError) as e:
         bs.bcast_schedule_shifted(p, root, 0, 0, 1, send, send)
     assert e.value.code == -6
+
+
+def test_more_blocks_than_one_launch_grid_holds():
+    # n above 65535: the per-block launches (arrival set-up, the reduction's last pass) go in slices
+    p, root, n = 5, 3, 70001
+    recv, send = oracle.schedule_table(p, root)
+    stats = check_broadcast(p, root, n, recv, send)
+    assert stats[:6].tolist() == [0] * 6 and stats[6] == (p - 1) * n and stats[7] == n - 1 + 3
+    value = contributions(p, n, 1)
+    result, rstats = check_reduce(p, root, n, recv, send, value)
+    with np.errstate(over="ignore"):
+        assert result.tolist() == value.sum(axis=1, dtype=np.uint64).tolist()
+    assert rstats[:6].tolist() == [0] * 6
