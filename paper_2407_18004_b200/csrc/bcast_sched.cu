@@ -182,6 +182,8 @@ struct SearchItem {
     uint16_t table;
 };
 
+constexpr int kLongFromRound = 2;               // searches wanted up to this round or beyond count as long
+
 // A queue serves a GROUP of consecutive rows of the tile whose threads drain it together:
 // the whole tile (kGroup = kThreads, the threads meet at block barriers) or one warp's 32
 // rows (kGroup = 32, the warp goes through pass, drain and flush on its own and meets no
@@ -191,9 +193,10 @@ struct GroupQueue {
     static constexpr int kGroupSize = kGroup;
     static constexpr int kSearchCapacity = 2 * kGroup;
     static constexpr int kCopyCapacity = 2 * kGroup;
-    SearchItem search[kSearchCapacity];
+    SearchItem search[kSearchCapacity];         // short searches from slot 0, long ones from the middle
     uint32_t copy[kCopyCapacity];               // src | dst << 9 | k << 18
-    int n_search;
+    int n_search;                               // short: highest wanted round below kLongFromRound
+    int n_long;
     int n_copy;
     __device__ __forceinline__ static void sync()
     {
@@ -201,7 +204,6 @@ struct GroupQueue {
     }
 };
 typedef GroupQueue<kThreads> TileQueue;
-typedef GroupQueue<32> WarpQueue;
 
 // Run the search for one item and drop the wanted entries into `row`.
 template <class Row, class Stats>
@@ -217,9 +219,12 @@ template <class Queue, class Tile, class Stats>
 __device__ __forceinline__ void push_search(const Geometry &g, Queue &queue, const SearchItem &it,
                                             const Tile &tile, Stats &stats)
 {
-    const int slot = atomicAdd(&queue.n_search, 1);
-    if (slot < Queue::kSearchCapacity) {
-        queue.search[slot] = it;
+    // a search runs until its highest wanted round; like lengths side by side keep a warp's lanes together
+    constexpr int kHalf = Queue::kSearchCapacity / 2;
+    const bool is_long = it.mask >= (1u << kLongFromRound);
+    const int slot = atomicAdd(is_long ? &queue.n_long : &queue.n_search, 1);
+    if (slot < kHalf) {
+        queue.search[(is_long ? kHalf : 0) + slot] = it;
     } else {
         resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
     }
@@ -332,10 +337,12 @@ __device__ __forceinline__ void drain_queue(const Geometry &g, Queue &queue, con
 {
     constexpr int kGroup = Queue::kGroupSize;
     const int member = threadIdx.x % kGroup;
-    const int n_search = min(queue.n_search, Queue::kSearchCapacity);
+    constexpr int kHalf = Queue::kSearchCapacity / 2;
+    const int n_short = min(queue.n_search, kHalf);
+    const int n_search = n_short + min(queue.n_long, kHalf);
     const int n_copy = min(queue.n_copy, Queue::kCopyCapacity);
     for (int i = member; i < n_search; i += kGroup) {
-        const SearchItem it = queue.search[i];
+        const SearchItem it = queue.search[i < n_short ? i : kHalf + (i - n_short)];
         // one call site: items for either table run the same instructions side by side
         resolve_item(g, it, it.table == 0 ? tile.recv_row(it.row) : tile.send_row(it.row), stats);
     }
@@ -624,7 +631,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
     for (int slot = 0; slot < tiles_per_block; ++slot) {
         const uint32_t t = group + (uint32_t)slot;
         if (t >= n_tiles) break;
-        if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
+        if (threadIdx.x == 0) { queue.n_search = 0; queue.n_long = 0; queue.n_copy = 0; }
         __syncthreads();                                   // descriptions built; previous tile flushed
         const uint32_t first = t * kThreads;
         const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
@@ -632,7 +639,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         tile_pass<Q>(tab, g, runs[slot], first_rank_of(first, rows), rows, tile, want_recv, want_send,
                      queue, ns);
         __syncthreads();
-        if (queue.n_search + queue.n_copy > 0) {           // the same for every thread
+        if (queue.n_search + queue.n_long + queue.n_copy > 0) {           // the same for every thread
             drain_queue(g, queue, tile, ns);
             __syncthreads();
         }
@@ -878,7 +885,7 @@ __device__ __forceinline__ void sweep_tables_of_p(const LevelTables &tab, const 
         for (int slot = 0; slot < kWarpsPerBlock; ++slot) {
             const uint32_t first = group + (uint32_t)slot * kThreads;
             if (first >= p) break;
-            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_copy = 0; }
+            if (threadIdx.x == 0) { queue.n_search = 0; queue.n_long = 0; queue.n_copy = 0; }
             row_viol[threadIdx.x] = 0u;
             __syncthreads();
             const ScratchTile tile{recv_tab, send_tab, first, p};
