@@ -85,6 +85,22 @@ def recorded_traffic(kernel: str, p, filename: str = "dram_traffic.txt"):
     return None
 
 
+def max_over_ranks(ms: float, world: int, device: str = "cuda") -> float:
+    """A time in ms as the maximum over all ranks of the job (replicas run side by side; the slowest counts)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank, steps: int, world: int, total_ms: float) -> float:
+    """Units all ranks processed in the timed steps per second of the slowest rank."""
+    return world * units_per_rank * steps / (total_ms * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock/throttle samples while the timed region runs."""
 
@@ -281,12 +297,9 @@ def run_ours(args):
     clocks = sampler.stop(t0, t1)
     per_step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
     total_ms = sum(per_step_ms)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world)
     ms_per_step = total_ms / args.steps
-    value = world * p * args.steps / (total_ms * 1e-3)
+    value = whole_job_value(p, args.steps, world, total_ms)
 
     # ---------------- end to end: host output tables through bcast_schedule_host
     e2e = None
@@ -312,11 +325,8 @@ def run_ours(args):
             ev1.record(stream)
             barrier()
             e2e_ms = ev0.elapsed_time(ev1)
-            if world > 1:
-                t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e2e_ms = float(t.item())
-            e2e = {"value": world * p * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+            e2e_ms = max_over_ranks(e2e_ms, world)
+            e2e = {"value": whole_job_value(p, e2e_steps, world, e2e_ms), "unit": UNIT,
                    "h2d_bytes_per_step": 0, "d2h_bytes_per_step": table_bytes, "steps": e2e_steps,
                    "ms_per_step": e2e_ms / e2e_steps,
                    "note": "bcast_schedule_host: tables land in pinned host memory; inputs are scalars"}
@@ -576,11 +586,8 @@ def run_other(args):
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
     total_ms = sum(per_step_ms)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = world * wl["units"] * args.steps / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, world)
+    value = whole_job_value(wl["units"], args.steps, world, total_ms)
 
     e2e = None
     if not args.no_e2e:
@@ -588,11 +595,8 @@ def run_other(args):
         torch.cuda.synchronize()
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
         e2e_ms = sum(timed(wl["e2e"], e2e_steps, False))
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * wl["units"] * e2e_steps / (e2e_ms * 1e-3), "unit": wl["unit"],
+        e2e_ms = max_over_ranks(e2e_ms, world)
+        e2e = {"value": whole_job_value(wl["units"], e2e_steps, world, e2e_ms), "unit": wl["unit"],
                "h2d_bytes_per_step": wl["h2d"], "d2h_bytes_per_step": wl["d2h"], "steps": e2e_steps,
                "ms_per_step": e2e_ms / e2e_steps}
     if rank != 0:

@@ -44,3 +44,17 @@ def test_reference_arm_other_modes():
         line = json.loads(out.stdout.strip().splitlines()[-1])
         assert line["impl"] == "reference" and line["metric"] == metric and line["value"] > 0
         assert line["cpu_baseline"]["kind"] == "oracle" and line["gpu_launches"] == 0
+
+
+def test_max_over_ranks_and_whole_job_value_two_gloo_ranks():
+    # the replicas of a multi-GPU run are timed as the slowest rank and counted together
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", "29733", os.path.join(ROOT, "tests", "dist_worker.py")]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    line = json.loads(lines[0])
+    assert line["world"] == 2 and line["total_ms"] == 15.0
+    assert abs(line["value"] - 2 * 1000 * 4 / 15e-3) < 1e-6
