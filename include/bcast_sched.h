@@ -10,8 +10,10 @@
  * Conventions for every entry point
  *  - Plain C types only.  "host" pointers are ordinary process memory; "device"
  *    pointers are CUDA global memory of the current device.  The caller owns
- *    every buffer; the library allocates nothing and keeps no state between
- *    calls (it is thread-safe).
+ *    every buffer and the library allocates nothing.  It is thread-safe and
+ *    keeps no state between calls, with two documented exceptions: the
+ *    process-wide launch-shape override (bcast_set_launch_shape) and the
+ *    built-in scratch array of bcast_verify_sweep_static.
  *  - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
  *    Device work is enqueued on it and the call returns without synchronising.
  *  - Return value: >= 0 on success (where stated, the value of q), otherwise a
@@ -22,6 +24,13 @@
  *    schedule of virtual rank (a - root + p) mod p.
  *  - Schedule entries are int32 in [-q, q-1] for rounds k = 0..q-1.  A negative
  *    entry names a block of an earlier phase (Algorithm 1 adds q per phase).
+ *  - The search of Algorithms 4 and 5 runs as a loop with an iteration cap far
+ *    above the bound of Lemma 6.  No p is known to reach the cap; should a
+ *    search ever do so, the entries it still owed read BCAST_UNRESOLVED in the
+ *    tables of bcast_schedule / bcast_allbroadcast_schedule / bcast_schedule_host
+ *    (BCAST_PAD in the rows of bcast_schedule_batch; bcast_schedule_shifted adds
+ *    its shift to the marker byte and does not preserve it), and
+ *    bcast_verify_sweep counts the event in fail_counts[7].
  */
 #ifndef BCAST_SCHED_H
 #define BCAST_SCHED_H
@@ -44,10 +53,18 @@ extern "C" {
 #define BCAST_ESTRIDE      -9   /* row_stride below 31                                  */
 #define BCAST_ESCRATCH     -10  /* scratch buffer too small for a single p of the range */
 #define BCAST_ETOOBIG      -11  /* p_hi above BCAST_STATIC_SWEEP_MAX_P                  */
+#define BCAST_EINVAL_SHAPE -12  /* not one of BCAST_SHAPE_*                             */
 
 #define BCAST_NONE         (-1)         /* bcast_round_block: nothing moves in this round */
 #define BCAST_PAD          INT32_MIN    /* filler of unused row entries in the batch form */
+#define BCAST_UNRESOLVED   (-128)       /* table entry a capped search never reached (see above) */
 #define BCAST_MAX_Q        31
+
+/* Launch shapes of the table kernel (bcast_set_launch_shape). */
+#define BCAST_SHAPE_AUTO     (-1)       /* chosen per call from an estimate (the default)          */
+#define BCAST_SHAPE_BLOCK      0        /* a block per tile, undecided entries searched per tile   */
+#define BCAST_SHAPE_WARPS      1        /* warps on their own, searches deferred to the block's end */
+#define BCAST_SHAPE_LOWFRAME   2        /* the same, low rounds looked up in a per-block table     */
 
 #define BCAST_STATIC_SWEEP_BYTES  (8u << 20)   /* built-in scratch of bcast_verify_sweep_static */
 #define BCAST_STATIC_SWEEP_MAX_P  65536        /* largest p_hi it accepts                       */
@@ -80,13 +97,23 @@ int bcast_skips(int32_t p, int32_t *skip_host);
  * the vector-store path).  Either table pointer may be NULL to skip that table,
  * not both.  An empty rank range and p = 1 (q = 0) succeed without a launch.
  * Asynchronous on cuda_stream.  Returns q.
- * The kernel has two launch shapes, chosen per call from an estimate of how
- * many entries of this p need the search of Algorithms 4 and 5; the environment
- * variable BCAST_LAUNCH_SHAPE=block|warps forces one (tuning, tests).  The
- * tables are the same either way.
+ * The kernel has three launch shapes, chosen per call from an estimate of how
+ * many entries of this p the closed forms leave to the search of Algorithms 4
+ * and 5 (bcast_set_launch_shape forces one).  The tables are the same in all.
  */
 int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end,
                    int32_t *recvblock_dev, int32_t *sendblock_dev, void *cuda_stream);
+
+/*
+ * Force a launch shape of the table kernel for all later calls of this process
+ * (tuning, and tests that run every shape on the same p): one of BCAST_SHAPE_*;
+ * BCAST_SHAPE_AUTO restores the per-call choice.  A shape a call cannot take
+ * (shifted tables, small q) falls back to one it can.  Until the first call of
+ * this function the environment variable BCAST_LAUNCH_SHAPE=block|warps|lowframe,
+ * read once, has the same effect.  Results never depend on the shape.  (No
+ * counterpart in the paper.)  Returns BCAST_OK or BCAST_EINVAL_SHAPE.
+ */
+int bcast_set_launch_shape(int shape);
 
 /*
  * bcast_schedule with the rows already prepared for n blocks, i.e. after the

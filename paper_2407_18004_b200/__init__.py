@@ -18,6 +18,8 @@ BCAST_NONE = -1
 BCAST_PAD = -(2 ** 31)
 BCAST_MAX_Q = 31
 BCAST_STATIC_SWEEP_MAX_P = 65536
+BCAST_UNRESOLVED = -128
+BCAST_SHAPE_AUTO, BCAST_SHAPE_BLOCK, BCAST_SHAPE_WARPS, BCAST_SHAPE_LOWFRAME = -1, 0, 1, 2
 
 _lib = None
 
@@ -37,6 +39,7 @@ def _load():
         lib.bcast_strerror.argtypes = [ctypes.c_int]
         lib.bcast_strerror.restype = ctypes.c_char_p
         lib.bcast_q.argtypes = [i32]
+        lib.bcast_set_launch_shape.argtypes = [ctypes.c_int]
         lib.bcast_skips.argtypes = [i32, vp]
         lib.bcast_schedule.argtypes = [i32, i32, i64, i64, vp, vp, vp]
         lib.bcast_schedule_host.argtypes = [i32, i32, i64, i64, vp, vp, vp, i64, vp]
@@ -88,6 +91,10 @@ def _stream(stream):
 # ------------------------------------------------------------------ host-only entry points
 def bcast_strerror(code: int) -> str:
     return _load().bcast_strerror(code).decode()
+
+
+def bcast_set_launch_shape(shape: int) -> int:
+    return _check(_load().bcast_set_launch_shape(shape))
 
 
 def bcast_q(p: int) -> int:

@@ -6,11 +6,12 @@ import subprocess
 import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = [os.path.join(_HERE, "csrc", "bcast_sched.cu"),
-           os.path.join(_HERE, "csrc", "bcast_simulate.cu")]
-HEADERS = [os.path.join(_HERE, "csrc", "schedule_core.cuh"),
-           os.path.join(_HERE, "csrc", "schedule_fast.cuh"),
-           os.path.join(os.path.dirname(_HERE), "include", "bcast_sched.h")]
+SOURCES = [os.path.join(_HERE, "csrc", name) for name in (
+    "table_q_top.cu", "table_q_high.cu", "table_q_mid.cu", "table_q_low.cu",
+    "bcast_sweep.cu", "bcast_sched.cu", "bcast_simulate.cu")]
+HEADERS = [os.path.join(_HERE, "csrc", name) for name in (
+    "schedule_core.cuh", "schedule_fast.cuh", "schedule_tile.cuh", "table_kernel.cuh", "host_util.h")]
+HEADERS.append(os.path.join(os.path.dirname(_HERE), "include", "bcast_sched.h"))
 LIBRARY = os.path.join(_HERE, "libbcast_sched.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -90,6 +90,11 @@ struct CountStats {
     { if (s.descents > q - 1 || s.steps > 2 * q + s.descents) s.over_bound = 1; }
 };
 
+// Value emitted for the rounds a search did not reach because it ran into its iteration cap
+// (BCAST_UNRESOLVED in the public header).  The cap lies far above Lemma 6's bound; no p is
+// known to reach it.
+constexpr int kUnresolvedEntry = -128;
+
 // State of the search of Algorithm 4 between two loop iterations.
 struct SearchState {
     uint32_t remaining;   // list of skip indices still linked
@@ -97,6 +102,8 @@ struct SearchState {
     uint32_t cand;        // part of the list the current call still has to scan
     uint32_t u;           // R - r'
     int b;                // baseblock of the rank
+    int k = 0;            // round the search is in (entries accepted so far)
+    uint32_t v = 0;       // R - s, s the processor accepted last (0 before the first: s = 2p never binds)
 };
 
 // Algorithm 5's set-up: all indices 0..q but the baseblock b, r' = 0, e = q.
@@ -164,15 +171,19 @@ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchS
     uint32_t pending = st.pending;
     uint32_t cand = st.cand;
     uint32_t u = st.u;                                    // R - r'
-    uint32_t v = 0;                                       // R - s
-    int k = 0;
-    uint32_t sk_k = 1u;                                   // skip[k]
-    uint32_t sk_k1 = skip_of(g, 1);                       // skip[k+1]
-    uint32_t m = 1u;                                      // max(skip[k], v+1)
+    uint32_t v = st.v;                                    // R - s
+    int k = st.k;
+    uint32_t sk_k = skip_of(g, k);                        // skip[k]
+    uint32_t sk_k1 = skip_of(g, k + 1 <= q ? k + 1 : q);  // skip[k+1]
+    uint32_t m = max(sk_k, v + 1u);                       // max(skip[k], v+1)
     int guard = 6 * q + 16;                               // never reached; keeps the loop finite
 
     while (true) {
-        if (--guard < 0) { stats.cap(); return; }
+        if (--guard < 0) {                                // mark what was still wanted and give up
+            stats.cap();
+            for (int kk = k; kk <= k_last; ++kk) emit(kk, kUnresolvedEntry);
+            return;
+        }
         int e;
         uint32_t bit, sk_e;
         bool accept;
@@ -275,6 +286,104 @@ __device__ __forceinline__ int recv_entry(const Geometry &g, uint32_t t, int k, 
     int value = 0;
     recv_search_fast(g, t, k, [&](int kk, int val) { if (kk == k) value = val; }, stats);
     return value;
+}
+
+// ---------------------------------------------------------------------------------------
+// The low rounds of the search, once per low state instead of once per rank.
+//
+// Let u >= 2 be what is left of R = p + r after its greedy digits at the levels >= L
+// (skip[q] = p first).  The search of Algorithms 4 and 5 descends on exactly those digits
+// before it accepts anything (search_from_digits), and from then on, until it first
+// returns past level L, every quantity it looks at is local to the levels below L: the
+// distance u, the list of indices < L without the baseblock (which is the lowest digit of
+// u, since u > 0), the skips below L and skip[k], skip[k+1] of the rounds it is in.  The
+// indices it accepts in that stretch are therefore a function of u alone for a given p, and
+// so is the number n of rounds it completes there.  When the stretch ends, the search
+// returns into the call that descended on the lowest digit j >= L of R and accepts j for
+// round n at once (R - r' >= skip[j] >= skip[n+1]), which gives one more round.
+//
+// The table of a frame packs that per u, a nibble per round k = 0..7: the accepted index
+// (< L <= 14), kLowFramePop for "the lowest digit of R at or above L" (value j - q, or the
+// rank's own baseblock when j = q), kLowFrameNone for rounds beyond.  u < 2 gives no rounds:
+// there the search stops descending above level L.
+//
+// The entries are built from one another.  Let x be the highest digit of u, u' = u - skip[x].
+// For u' >= 2 the search first descends on x and is then in the same situation one frame
+// down, so its first rounds are the entry of u'; where that stretch ends it returns to x
+// and accepts it.  (u' = 1: x is accepted for round 0 at once.  u' = 0: x is the baseblock
+// and not in the list.)  Only what follows needs the search itself, started from the state
+// that prefix leaves: back in the outermost call, scanning below x.  A block fills the
+// table level by level (all u with the same highest digit side by side, a barrier between
+// the levels).
+constexpr uint32_t kLowFramePop = 14u;
+constexpr uint32_t kLowFrameNone = 15u;
+constexpr int kLowFrameRounds = 8;
+
+// Entry of u, skip[x] <= u < skip[x+1], given the entries of every smaller u.
+__device__ __forceinline__ uint32_t low_frame_entry(const Geometry &g, int L, const uint32_t *table, int x,
+                                                    uint32_t u)
+{
+    constexpr uint32_t kNone = 0xffffffffu;
+    if (u < 2u) return kNone;
+    const uint32_t sk_x = skip_of(g, x);
+    const uint32_t left = u - sk_x;                        // u'
+    uint32_t packed = kNone;
+    uint32_t taken = 0u;                                   // indices accepted so far
+    int rounds = 0;
+    int b = x;                                             // left = 0: x is the baseblock
+    if (left >= 1u) {
+        // the baseblock: lowest digit of u, i.e. of u'
+        uint32_t rem = left;
+        for (int k = x - 1; k >= 0; --k) {
+            const uint32_t s = skip_of(g, k);
+            if (rem >= s) { rem -= s; if (rem == 0u) { b = k; break; } }
+        }
+        if (left >= 2u) {
+            const uint32_t prefix = table[left];
+            while (rounds < kLowFrameRounds) {
+                const uint32_t nib = (prefix >> (4 * rounds)) & 15u;
+                if (nib >= kLowFramePop) break;
+                taken |= 1u << nib;
+                ++rounds;
+            }
+            if (rounds == kLowFrameRounds) return prefix;
+            packed = prefix | (kNone << (4 * rounds));      // the prefix's rounds, nothing beyond yet
+        }
+        packed = (packed & ~(15u << (4 * rounds))) | ((uint32_t)x << (4 * rounds));    // x accepted
+        taken |= 1u << x;
+        if (++rounds == kLowFrameRounds) return packed;
+    }
+    SearchState s;
+    s.b = b;
+    s.remaining = ((1u << L) - 1u) & ~(1u << b) & ~taken;
+    s.pending = 0u;
+    s.cand = s.remaining & ((1u << x) - 1u);
+    s.u = u;
+    s.k = rounds;
+    s.v = left >= 1u ? left : 0u;
+    bool capped = false;
+    NoStats ns;
+    recv_search_run(g, s, kLowFrameRounds - 1, [&](int k, int val) {
+        if (val == kUnresolvedEntry) { capped = true; return; }
+        packed = (packed & ~(15u << (4 * k))) | ((uint32_t)(val + g.q) << (4 * k));
+        rounds = k + 1;
+    }, ns);
+    if (capped) return kNone;
+    if (rounds < kLowFrameRounds)
+        packed = (packed & ~(15u << (4 * rounds))) | (kLowFramePop << (4 * rounds));
+    return packed;
+}
+
+// Fills table[0 .. min(skip[L], capacity)) ; called by every thread of the block.
+__device__ __forceinline__ void low_frame_build(const Geometry &g, int L, uint32_t *table, uint32_t capacity)
+{
+    const uint32_t n_states = min(skip_of(g, L), capacity);
+    if (threadIdx.x < 2u) table[threadIdx.x] = 0xffffffffu;
+    for (int x = 1; x < L; ++x) {
+        const uint32_t lo = skip_of(g, x), hi = min(skip_of(g, x + 1), n_states);
+        for (uint32_t u = lo + threadIdx.x; u < hi; u += blockDim.x) table[u] = low_frame_entry(g, L, table, x, u);
+        __syncthreads();
+    }
 }
 
 }  // namespace bcast

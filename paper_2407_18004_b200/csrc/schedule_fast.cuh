@@ -350,16 +350,19 @@ __device__ __forceinline__ void build_tile_runs(const LevelTables &tab, const Le
 }
 
 // The high-level entries of the rank in row `row` from its run's description; returns
-// the walk state entering level kSharedFrom-1 for that rank.
+// the walk state entering level kSharedFrom-1 for that rank and, on request, the first row
+// past the rank's run.
 template <int Q, class Row>
 __device__ __forceinline__ WalkState<typename WalkInt<Q>::type>
-apply_tile_runs(const TileRuns<typename WalkInt<Q>::type> &runs, int row, Row recv_row, Row send_row)
+apply_tile_runs(const TileRuns<typename WalkInt<Q>::type> &runs, int row, Row recv_row, Row send_row,
+                int *run_end = nullptr)
 {
     typedef typename WalkInt<Q>::type Int;
     int run = 0;
 #pragma unroll
     for (int i = 1; i < kMaxRuns; ++i) run += row >= runs.start[i] ? 1 : 0;
     const int t = row - runs.start[run];
+    if (run_end != nullptr) *run_end = runs.start[run + 1];     // unused entries hold the row count
     WalkState<Int> s = runs.state[run];
     s.rp += (Int)t;
     s.A += (Int)t;

@@ -30,3 +30,14 @@ def load_golden(name):
 @pytest.fixture(scope="session")
 def golden():
     return load_golden
+
+
+@pytest.fixture
+def forced_shape():
+    """forced_shape("block" | "warps" | "lowframe" | "auto") forces a launch shape of the table kernel for
+    the rest of the test; the per-call choice is restored afterwards."""
+    import paper_2407_18004_b200 as bs
+    names = {"auto": bs.BCAST_SHAPE_AUTO, "block": bs.BCAST_SHAPE_BLOCK, "warps": bs.BCAST_SHAPE_WARPS,
+             "lowframe": bs.BCAST_SHAPE_LOWFRAME}
+    yield lambda name: bs.bcast_set_launch_shape(names[name])
+    bs.bcast_set_launch_shape(bs.BCAST_SHAPE_AUTO)

@@ -1,6 +1,5 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle,
 bit for bit, on the same seeded inputs."""
-import os
 
 import numpy as np
 import pytest
@@ -279,10 +278,9 @@ def test_schedule_host_chunks():
 # ------------------------------------------------------------------ Algorithm 7: all-broadcast tables
 @pytest.mark.parametrize("p,rank", [(2, 1), (17, 5), (1000, 0), (1000, 999), (1000, 417), (5000, 1234),
                                     (70001, 69999), (2 ** 16 + 1, 3), (2 ** 17 - 1, 77)])
-@pytest.mark.parametrize("shape", ["auto", "block", "warps"])
-def test_allbroadcast_tables(monkeypatch, shape, p, rank):
-    if shape != "auto":
-        monkeypatch.setenv("BCAST_LAUNCH_SHAPE", shape)        # both launch shapes of the table kernel
+@pytest.mark.parametrize("shape", ["auto", "block", "warps", "lowframe"])
+def test_allbroadcast_tables(forced_shape, shape, p, rank):
+    forced_shape(shape)                                        # every launch shape of the table kernel
     orecv, osend = oracle.allbroadcast_schedule(p, rank)
     recv, send = bs.allbroadcast_schedule(p, rank)
     torch.cuda.synchronize()
@@ -295,17 +293,15 @@ def test_allbroadcast_tables(monkeypatch, shape, p, rank):
         assert_equal(f"sendblocks[{lo}:{hi}]", send.cpu().numpy(), osend[lo:hi])
 
 
-def test_allbroadcast_large_p_is_the_reversed_broadcast_table():
+def test_allbroadcast_large_p_is_the_reversed_broadcast_table(forced_shape):
     """p = 2^20+1: row j of processor r's tables is row (r - j) mod p of the root-0 tables."""
     p, rank = workloads.P_MEDIUM, 777777
     recv0, send0 = bs.schedule(p)
     recv, send = bs.allbroadcast_schedule(p, rank)
-    os.environ["BCAST_LAUNCH_SHAPE"] = "warps"             # the other shape too (its deferred queue overflows here)
-    try:
+    for shape in ("warps", "block"):                       # the other shapes too (the deferred queue overflows here)
+        forced_shape(shape)
         recv_w, send_w = bs.allbroadcast_schedule(p, rank)
-    finally:
-        del os.environ["BCAST_LAUNCH_SHAPE"]
-    assert bool((recv_w == recv).all()) and bool((send_w == send).all())
+        assert bool((recv_w == recv).all()) and bool((send_w == send).all()), shape
     torch.cuda.synchronize()
     idx = (rank - torch.arange(p, device="cuda")) % p
     assert bool((recv == recv0[idx]).all()) and bool((send == send0[idx]).all())
@@ -392,13 +388,13 @@ def test_table_kernel_against_batch_kernel_at_scale(p, root):
 
 
 # ------------------------------------------------------------------ both launch shapes of the table kernel
-@pytest.mark.parametrize("shape", ["block", "warps"])
+@pytest.mark.parametrize("shape", ["block", "warps", "lowframe"])
 @pytest.mark.parametrize("p,root", [(1000, 0), (5000, 1234), (2 ** 16 + 1, 7), (300007, 299999), (2 ** 20 + 1, 0),
-                                    (2 ** 20 - 1, 5)])
-def test_both_launch_shapes_full_tables(monkeypatch, shape, p, root):
-    """The library picks the launch shape from an estimate; forced either way, on p with many and with few
+                                    (2 ** 20 - 1, 5), (3 * 2 ** 18, 11), (999983, 500000)])
+def test_every_launch_shape_full_tables(forced_shape, shape, p, root):
+    """The library picks the launch shape from an estimate; forced each way, on p with many and with few
     undecided entries (the block's deferred queue overflows at p = 2^20 + 1), the tables equal the oracle's."""
-    monkeypatch.setenv("BCAST_LAUNCH_SHAPE", shape)
+    forced_shape(shape)
     recv, send = gpu_tables(p, root)
     orecv, osend = oracle.schedule_table(p, root)
     assert_equal("recvblock (%s)" % shape, recv, orecv)
