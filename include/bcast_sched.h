@@ -65,6 +65,8 @@ extern "C" {
 #define BCAST_SHAPE_BLOCK      0        /* a block per tile, undecided entries searched per tile   */
 #define BCAST_SHAPE_WARPS      1        /* warps on their own, searches deferred to the block's end */
 #define BCAST_SHAPE_LOWFRAME   2        /* the same, low rounds looked up in a per-block table     */
+#define BCAST_SHAPE_WARPS_TIGHT 3       /* BCAST_SHAPE_WARPS with next to no queue space: for tests */
+                                        /* of the path that recomputes a group whose queues ran full */
 
 #define BCAST_STATIC_SWEEP_BYTES  (8u << 20)   /* built-in scratch of bcast_verify_sweep_static */
 #define BCAST_STATIC_SWEEP_MAX_P  65536        /* largest p_hi it accepts                       */
@@ -109,7 +111,7 @@ int bcast_schedule(int32_t p, int32_t root, int64_t rank_begin, int64_t rank_end
  * (tuning, and tests that run every shape on the same p): one of BCAST_SHAPE_*;
  * BCAST_SHAPE_AUTO restores the per-call choice.  A shape a call cannot take
  * (shifted tables, small q) falls back to one it can.  Until the first call of
- * this function the environment variable BCAST_LAUNCH_SHAPE=block|warps|lowframe,
+ * this function the environment variable BCAST_LAUNCH_SHAPE=block|warps|lowframe|tight,
  * read once, has the same effect.  Results never depend on the shape.  (No
  * counterpart in the paper.)  Returns BCAST_OK or BCAST_EINVAL_SHAPE.
  */

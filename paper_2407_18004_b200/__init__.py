@@ -19,7 +19,7 @@ BCAST_PAD = -(2 ** 31)
 BCAST_MAX_Q = 31
 BCAST_STATIC_SWEEP_MAX_P = 65536
 BCAST_UNRESOLVED = -128
-BCAST_SHAPE_AUTO, BCAST_SHAPE_BLOCK, BCAST_SHAPE_WARPS, BCAST_SHAPE_LOWFRAME = -1, 0, 1, 2
+BCAST_SHAPE_AUTO, BCAST_SHAPE_BLOCK, BCAST_SHAPE_WARPS, BCAST_SHAPE_LOWFRAME, BCAST_SHAPE_WARPS_TIGHT = -1, 0, 1, 2, 3
 
 _lib = None
 

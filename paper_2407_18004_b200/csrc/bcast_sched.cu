@@ -274,7 +274,7 @@ static bool undecided_at_most(const LevelTables &tab, int64_t p, int q, double m
 
 // A forced launch shape of the table kernel (tuning, and the tests, which run every shape on the
 // same p): process-wide, BCAST_SHAPE_AUTO unless bcast_set_launch_shape() or, at its first use, the
-// environment variable BCAST_LAUNCH_SHAPE=block|warps|lowframe says otherwise.
+// environment variable BCAST_LAUNCH_SHAPE=block|warps|lowframe|tight says otherwise.
 static std::atomic<int> &forced_shape()
 {
     static std::atomic<int> forced([] {
@@ -283,6 +283,7 @@ static std::atomic<int> &forced_shape()
         if (strcmp(v, "block") == 0) return BCAST_SHAPE_BLOCK;
         if (strcmp(v, "warps") == 0) return BCAST_SHAPE_WARPS;
         if (strcmp(v, "lowframe") == 0) return BCAST_SHAPE_LOWFRAME;
+        if (strcmp(v, "tight") == 0) return BCAST_SHAPE_WARPS_TIGHT;
         return BCAST_SHAPE_AUTO;
     }());
     return forced;
@@ -356,9 +357,10 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
 
 int bcast_set_launch_shape(int shape)
 {
-    if (shape < BCAST_SHAPE_AUTO || shape > BCAST_SHAPE_LOWFRAME) return BCAST_EINVAL_SHAPE;
+    if (shape < BCAST_SHAPE_AUTO || shape > BCAST_SHAPE_WARPS_TIGHT) return BCAST_EINVAL_SHAPE;
     static_assert(BCAST_SHAPE_BLOCK == kShapeBlockPerTile && BCAST_SHAPE_WARPS == kShapeWarps &&
-                  BCAST_SHAPE_LOWFRAME == kShapeWarpsLowFrame, "public and internal shape numbers agree");
+                  BCAST_SHAPE_LOWFRAME == kShapeWarpsLowFrame && BCAST_SHAPE_WARPS_TIGHT == kShapeWarpsTight,
+                  "public and internal shape numbers agree");
     forced_shape().store(shape, std::memory_order_relaxed);
     return BCAST_OK;
 }

@@ -366,9 +366,10 @@ struct SharedTile {
 // there).  What is undecided is queued per group of kWarpsPerBlock tiles, and when the
 // group's tiles are out the whole block works the queues off, storing every entry straight
 // into the output table, over the placeholder:
-//   1. searches (DeferredItem): the receive schedule of a virtual rank is searched up to
-//      the highest round wanted; kind 0 fills receive entries of the rank's own row,
-//      kind 1 one send entry of a row whose to-processor the rank is;
+//   1. searches (DeferredItem): the receive schedule of a virtual rank is searched up to a round k;
+//      kind 0 writes the receive entries of the rank's own row for every round up to k (the search
+//      yields them all, and those the pass had decided are the same), kind 1 the send entry of
+//      round k of a row whose to-processor the rank is;
 //   2. after a barrier, fix-ups: a send entry whose to-processor is a row of the same
 //      group is that row's receive entry (Section 2.3), final in the output table by
 //      then, and is copied from there.
@@ -376,12 +377,10 @@ struct SharedTile {
 // per warp even fewer.)
 struct DeferredItem {
     uint32_t rank;                                         // virtual rank whose receive schedule is searched
-    uint32_t row_kind;                                     // output row relative to the group | kind << 31
-    uint32_t mask;                                         // rounds wanted
-    uint32_t reserved;
-};
+    uint32_t what;                                         // output row relative to the group | k << 11 | kind << 16
+};                                                         // kind 0: every round up to k; kind 1: round k alone
 
-constexpr int kDeferredCapacity = 160;
+constexpr int kDeferredCapacity = 384;
 constexpr int kFixupCapacity = 1024;
 constexpr int kGroupRows = kWarpsPerBlock * kThreads;  // rows of a group of tiles: fix-ups hold a row in 11 bits
 constexpr int kLowFrameTiles = 64;                     // most tiles of a block that builds the table of low states
@@ -391,6 +390,8 @@ constexpr int kLowFrameStates = 512;                   // skip[kSharedFrom] <= 2
 constexpr int kShapeBlockPerTile = 0;                  // the block meets after every tile and drains its queues
 constexpr int kShapeWarps = 1;                         // warps on their own, searches deferred to the group's end
 constexpr int kShapeWarpsLowFrame = 2;                 // the same, undecided low rounds from the table of low states
+constexpr int kShapeWarpsTight = 3;                    // kShapeWarps with room for kTightCapacity queue entries (tests)
+constexpr int kTightCapacity = 8;
 constexpr int kDescWarpsFromQ = 16;                    // smallest q with a descending-rows kernel of that shape
 
 struct DeferredQueue {
@@ -400,6 +401,7 @@ struct DeferredQueue {
     uint32_t need_recv[kWarpsPerBlock][32];                // per warp and row of its slice: rounds to search
     int n_items[2];                                        // counters for groups of tiles taken in turn
     int n_fixups[2];
+    uint32_t overflow;                                     // groups of the block (a bit each) that found a queue full
 };
 
 union QueueStorage {
@@ -407,24 +409,71 @@ union QueueStorage {
     DeferredQueue deferred;                                // the group's deferred work
 };
 
+// Both rows of `rows` consecutive output rows by the search alone (Algorithms 4-6 per rank,
+// as for independent queries), written straight into the tables.  Slow: the way out for a
+// group of tiles whose queues overflowed, run at the block's end, apart from the code of the pass.
+// index0: output index of the first row (row x holds virtual rank (index - anchor) mod p, or
+// (anchor - index) mod p for descending rows); recv/send point at that row (either may be null).
+struct IntRow {
+    int32_t *row;
+    __device__ __forceinline__ void operator()(int k, int val) const { row[k] = val; }
+};
+
+static __device__ __forceinline__ void rows_by_search(uint32_t p, uint32_t anchor, uint32_t index0, int descending,
+                                                   uint32_t rows, int32_t *recv, int32_t *send)
+{
+    const Geometry g = make_geometry(p);
+    NoStats ns;
+    for (uint32_t i = threadIdx.x; i < rows; i += blockDim.x) {
+        const uint32_t index = index0 + i;
+        const uint32_t r = descending ? (anchor >= index ? anchor - index : anchor + (p - index))
+                                      : (index >= anchor ? index - anchor : index + (p - anchor));
+        rank_rows(g, r, IntRow{recv + (size_t)i * g.q}, IntRow{send + (size_t)i * g.q}, recv != nullptr,
+                  send != nullptr, ns);
+    }
+}
+
 // Search for one deferred item; emit(table, row, k, value) receives every wanted entry
 // (table 0 = receive, 1 = send; row relative to the group's first row).
 template <class Emit>
 __device__ __forceinline__ void resolve_deferred(const Geometry &g, const DeferredItem &it, Emit emit)
 {
-    const uint32_t row = it.row_kind & 0x7fffffffu;
-    const int table = (int)(it.row_kind >> 31);
-    const uint32_t mask = it.mask;
+    const uint32_t row = it.what & 2047u;
+    const int k_last = (int)((it.what >> 11) & 31u);
+    const bool one_send = (it.what >> 16) != 0u;
     NoStats ns;
-    recv_search_fast(g, it.rank, 31 - __clz(mask), [&](int k, int val) {
-        if ((mask >> k) & 1u) emit(table, row, k, val);
+    recv_search_fast(g, it.rank, k_last, [&](int k, int val) {
+        if (!one_send) emit(0, row, k, val);
+        else if (k == k_last) emit(1, row, k, val);
     }, ns);
+}
+
+// A table word of low_frame_entry as schedule values: byte k of the pair holds the value of
+// round k (index - q; the lowest shared digit j_high - q where the search returned past the
+// low levels), and bit k of the result says whether the table has that round at all.
+template <int Q>
+__device__ __forceinline__ uint32_t low_frame_values(uint32_t word, int j_high, uint32_t &rounds_0_3,
+                                                     uint32_t &rounds_4_7)
+{
+    const uint32_t even = word & 0x0f0f0f0fu, odd = (word >> 4) & 0x0f0f0f0fu;     // nibbles 0,2,4,6 / 1,3,5,7
+    uint32_t lo = __byte_perm(even, odd, 0x5140), hi = __byte_perm(even, odd, 0x7362);
+    const uint32_t none_lo = __vcmpeq4(lo, 0x0f0f0f0fu), none_hi = __vcmpeq4(hi, 0x0f0f0f0fu);
+    const uint32_t pop_lo = __vcmpeq4(lo, 0x0e0e0e0eu), pop_hi = __vcmpeq4(hi, 0x0e0e0e0eu);
+    const uint32_t j4 = (uint32_t)j_high * 0x01010101u;
+    lo = (lo & ~pop_lo) | (j4 & pop_lo);
+    hi = (hi & ~pop_hi) | (j4 & pop_hi);
+    constexpr uint32_t kMinusQ = (uint32_t)((-Q) & 0xff) * 0x01010101u;
+    rounds_0_3 = add_bytes(lo, kMinusQ);
+    rounds_4_7 = add_bytes(hi, kMinusQ);
+    // one bit per byte: 0x80 of each byte gathered into bits 0..3
+    const uint32_t have_lo = ~none_lo & 0x80808080u, have_hi = ~none_hi & 0x80808080u;
+    return ((have_lo * 0x00204081u) >> 28) | (((have_hi * 0x00204081u) >> 28) << 4);
 }
 
 // Undecided low rounds from the table of the search's low states (low_frame_entry): the
 // rank's own receive entries from its own state u_low, and its send entries from the state
 // of its to-processor where that is a rank of the same run (same digits at the levels
-// >= kSharedFrom, u_low + skip[k] left below them).  Straight-line code over the rounds.
+// >= kSharedFrom, u_low + skip[k] left below them).
 template <int Q, class Row>
 __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const uint32_t *low_frame,
                                                   uint32_t u_low, int j_high, uint32_t ahead, uint32_t run_end,
@@ -432,30 +481,35 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
                                                   uint32_t &send_flags)
 {
     constexpr uint32_t kLowMask = (1u << kLowFrameRounds) - 1u;
-    if (((recv_flags | send_flags) & kLowMask) == 0u) return;
-    const uint32_t word = low_frame[u_low];
+    {   // receive entries: straight-line, a predicated byte store per round
+        uint32_t v03, v47;
+        const uint32_t have = low_frame_values<Q>(low_frame[u_low], j_high, v03, v47);
+        const uint32_t take = recv_flags & have & kLowMask;
 #pragma unroll
-    for (int k = 0; k < kLowFrameRounds && k < Q; ++k) {
-        const uint32_t bit = 1u << k;
-        const uint32_t nib = (word >> (4 * k)) & 15u;
-        if ((recv_flags & bit) != 0u && nib <= kLowFramePop) {
-            recv_row(k, (nib == kLowFramePop ? j_high : (int)nib) - Q);
-            recv_flags ^= bit;
-        }
-        if ((send_flags & bit) != 0u && ahead + tab.skip[k] < run_end) {
-            const uint32_t nib_t = (low_frame[u_low + tab.skip[k]] >> (4 * k)) & 15u;
-            if (nib_t <= kLowFramePop) {
-                send_row(k, (nib_t == kLowFramePop ? j_high : (int)nib_t) - Q);
-                send_flags ^= bit;
+        for (int k = 0; k < kLowFrameRounds && k < Q; ++k)
+            if ((take >> k) & 1u) recv_row(k, (int)(int8_t)((k < 4 ? v03 : v47) >> (8 * (k & 3))));
+        recv_flags ^= take;
+    }
+    // send entries: at most four per rank (Theorem 3), one table word each
+    uint32_t todo = send_flags & kLowMask;
+    while (todo != 0u) {
+        const int k = __ffs(todo) - 1;
+        todo &= todo - 1u;
+        const uint32_t skip_k = skip_of(make_geometry(tab.skip[Q]), k);
+        if (ahead + skip_k < run_end) {
+            const uint32_t nib = (low_frame[u_low + skip_k] >> (4 * k)) & 15u;
+            if (nib <= kLowFramePop) {
+                send_row(k, (nib == kLowFramePop ? j_high : (int)nib) - Q);
+                send_flags ^= 1u << k;
             }
         }
     }
 }
 
 // The closed-form pass of one warp's 32 rows of a tile (lane l owns row 32*warp + l).  Rounds
-// the pass cannot decide are looked up (low_frame, if given) or queued; when a queue is full
-// the lane runs the search itself and puts the entries into the staged rows, which are not
-// flushed yet.  group_row0: the tile's first output row relative to the group; group_rows:
+// the pass cannot decide are looked up (low_frame, if given) or queued; a full queue drops the
+// item and marks the group, whose rows the caller then computes again by the search alone.
+// capacity_cut takes room away from the queues (0 normally; the tests' tight shape).  group_row0: the tile's first output row relative to the group; group_rows:
 // output rows of the group.
 template <int Q, bool desc, class Tile>
 __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry &g,
@@ -463,7 +517,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
                                           uint32_t r_first, uint32_t rows, uint32_t group_row0,
                                           uint32_t group_rows, const Tile &tile,
                                           bool want_recv, bool want_send, DeferredQueue &dq, int phase,
-                                          const uint32_t *low_frame)
+                                          uint32_t group_bit, int capacity_cut, const uint32_t *low_frame)
 {
     // index: the thread's row of the staged tile = its output row within the tile.  The ranks of a tile
     // ascend with the row, or descend (Algorithm 7's tables); `ahead` is the thread's place counted from
@@ -486,13 +540,10 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
 
     auto defer = [&](const DeferredItem &it) {
         const int slot = atomicAdd(&dq.n_items[phase], 1);
-        if (slot < kDeferredCapacity) {
+        if (slot < kDeferredCapacity - capacity_cut) {
             dq.items[slot] = it;
         } else {
-            resolve_deferred(g, it, [&](int table, uint32_t row, int k, int val) {
-                const uint32_t in_tile = row - group_row0;
-                if (table == 0) tile.recv_row(in_tile)(k, val); else tile.send_row(in_tile)(k, val);
-            });
+            atomicOr(&dq.overflow, group_bit);             // the group's rows are redone by rows_by_search
         }
     };
     // Algorithm 6 could not decide round k of the send row of tile row `row` (virtual rank rr): the entry
@@ -505,14 +556,14 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
         const bool in_group = desc ? out_row >= skip_k : out_row + skip_k < group_rows;
         if (want_recv && in_group) {
             const int slot = atomicAdd(&dq.n_fixups[phase], 1);
-            if (slot < kFixupCapacity) {
+            if (slot < kFixupCapacity - capacity_cut * (kFixupCapacity / kDeferredCapacity)) {
                 dq.fixups[slot] = (uint16_t)(out_row | ((uint32_t)k << 11));
                 return;
             }
         }
         uint32_t t = rr + skip_k;
         if (t >= g.p) t -= g.p;
-        defer(DeferredItem{t, out_row | 0x80000000u, 1u << k, 0u});
+        defer(DeferredItem{t, out_row | ((uint32_t)k << 11) | (1u << 16)});
     };
 
     uint32_t recv_flags = 0, send_flags = 0;
@@ -520,15 +571,22 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     if constexpr (Q >= kSharedFrom + 2) {
         shared = runs.n_runs > 0;                          // the same for the whole block
         if (shared) {
-            int run_end = 0;
-            auto st = apply_tile_runs<Q>(runs, (int)ahead, recv_row, send_row, &run_end);
-            const uint32_t u_low = (uint32_t)st.rp;         // what the levels >= kSharedFrom leave of the rank
-            const int j_high = st.j;                       // its lowest digit at those levels (Q: none)
+            auto st = apply_tile_runs<Q>(runs, (int)ahead, recv_row, send_row);
             closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
             closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
-            if (low_frame != nullptr && j_high < Q)
-                low_frame_lookups<Q>(tab, low_frame, u_low, j_high, ahead, (uint32_t)run_end, recv_row, send_row,
-                                     recv_flags, send_flags);
+            constexpr uint32_t kLowMask = (1u << kLowFrameRounds) - 1u;
+            if (low_frame != nullptr && __any_sync(0xffffffffu, ((recv_flags | send_flags) & kLowMask) != 0u)) {
+                // the rank's state below the shared levels, read again from its run's description
+                // rather than kept in registers across the pass
+                int run = 0;
+#pragma unroll
+                for (int i = 1; i < kMaxRuns; ++i) run += (int)ahead >= runs.start[i] ? 1 : 0;
+                const uint32_t u_low = (uint32_t)runs.state[run].rp + (ahead - (uint32_t)runs.start[run]);
+                const int j_high = runs.state[run].j;      // lowest digit at the shared levels (Q: none)
+                if (j_high < Q)
+                    low_frame_lookups<Q>(tab, low_frame, u_low, j_high, ahead, (uint32_t)runs.start[run + 1],
+                                         recv_row, send_row, recv_flags, send_flags);
+            }
             // entries of the high levels that the description left undecided (at most 32, one per
             // lane); each warp takes those of its own rows, once their placeholders are written
             __syncwarp();
@@ -565,7 +623,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     }
     __syncwarp();
     const uint32_t mine = (want_recv ? recv_flags : 0u) | need_recv[lane];
-    if (mine != 0u) defer(DeferredItem{r, group_row0 + index, mine, 0u});
+    if (mine != 0u) defer(DeferredItem{r, (group_row0 + index) | ((uint32_t)(31 - __clz(mine)) << 11)});
 }
 
 }  // namespace bcast

@@ -67,8 +67,10 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         constexpr bool desc = kDescWarps;
         DeferredQueue &dq = queues.deferred;
         if (threadIdx.x < 2) { dq.n_items[threadIdx.x] = 0; dq.n_fixups[threadIdx.x] = 0; }
+        if (threadIdx.x == 2) dq.overflow = 0u;
         // the low rounds of the search for every low state of this p, when the host expects
         // enough undecided entries to pay for it
+        const int capacity_cut = shape == kShapeWarpsTight ? kDeferredCapacity - kTightCapacity : 0;
         const uint32_t *low_frame = nullptr;
         if constexpr (Q >= kSharedFrom + 2) {
             if (shape == kShapeWarpsLowFrame) {            // the same for the whole block
@@ -90,7 +92,8 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
                 const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
                 const SharedTile<Q> tile{recv_bytes, send_bytes, rows, false};
                 warp_pass<Q, desc>(tab, g, runs[slot], first_rank_of(first, rows), rows, (uint32_t)slot * kThreads,
-                                   group_rows, tile, want_recv, want_send, dq, phase, low_frame);
+                                   group_rows, tile, want_recv, want_send, dq, phase, 1u << (done / kWarpsPerBlock),
+                                   capacity_cut, low_frame);
                 __syncwarp();                              // the slice is staged
                 const uint32_t my_first = (uint32_t)warp * 32u;
                 if (my_first < rows) {
@@ -104,8 +107,9 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             }
             __syncthreads();                               // every slice of the group is out; now its searches
             const size_t group_base = (size_t)group * kThreads * (size_t)Q;
-            const int n_items = min(dq.n_items[phase], kDeferredCapacity);
-            const int n_fixups = min(dq.n_fixups[phase], kFixupCapacity);
+            const int n_items = min(dq.n_items[phase], kDeferredCapacity - capacity_cut);
+            const int n_fixups = min(dq.n_fixups[phase],
+                                     kFixupCapacity - capacity_cut * (kFixupCapacity / kDeferredCapacity));
             for (int i = threadIdx.x; i < n_items; i += kThreads) {
                 resolve_deferred(g, dq.items[i], [&](int table, uint32_t row, int k, int val) {
                     int32_t *out = table == 0 ? recv_out : send_out;
@@ -126,6 +130,20 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             if (threadIdx.x < 2) {
                 if (threadIdx.x == 0) dq.n_items[phase ^ 1] = 0; else dq.n_fixups[phase ^ 1] = 0;
             }
+        }
+        // groups that found a queue full (bit = number of the group within the block): their rows
+        // again, by the search alone
+        __syncthreads();
+        uint32_t redo = dq.overflow;
+        while (redo != 0u) {                               // the same for the whole block
+            const uint32_t first_tile = block_first_tile + (uint32_t)(__ffs(redo) - 1) * kWarpsPerBlock;
+            redo &= redo - 1u;
+            const uint32_t first = first_tile * kThreads;
+            const uint32_t left = (uint32_t)tiles_per_block * kThreads - (first - block_first_tile * kThreads);
+            const uint32_t rows = min(min((uint32_t)kGroupRows, left), n_ranks - first);
+            const size_t at = (size_t)first * (size_t)Q;
+            rows_by_search(p, anchor, row_begin + first, descending, rows,
+                           want_recv ? recv_out + at : nullptr, want_send ? send_out + at : nullptr);
         }
         return;
     }

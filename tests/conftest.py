@@ -34,10 +34,10 @@ def golden():
 
 @pytest.fixture
 def forced_shape():
-    """forced_shape("block" | "warps" | "lowframe" | "auto") forces a launch shape of the table kernel for
+    """forced_shape("block" | "warps" | "lowframe" | "tight" | "auto") forces a launch shape of the table kernel for
     the rest of the test; the per-call choice is restored afterwards."""
     import paper_2407_18004_b200 as bs
     names = {"auto": bs.BCAST_SHAPE_AUTO, "block": bs.BCAST_SHAPE_BLOCK, "warps": bs.BCAST_SHAPE_WARPS,
-             "lowframe": bs.BCAST_SHAPE_LOWFRAME}
+             "lowframe": bs.BCAST_SHAPE_LOWFRAME, "tight": bs.BCAST_SHAPE_WARPS_TIGHT}
     yield lambda name: bs.bcast_set_launch_shape(names[name])
     bs.bcast_set_launch_shape(bs.BCAST_SHAPE_AUTO)

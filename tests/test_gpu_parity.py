@@ -278,7 +278,7 @@ def test_schedule_host_chunks():
 # ------------------------------------------------------------------ Algorithm 7: all-broadcast tables
 @pytest.mark.parametrize("p,rank", [(2, 1), (17, 5), (1000, 0), (1000, 999), (1000, 417), (5000, 1234),
                                     (70001, 69999), (2 ** 16 + 1, 3), (2 ** 17 - 1, 77)])
-@pytest.mark.parametrize("shape", ["auto", "block", "warps", "lowframe"])
+@pytest.mark.parametrize("shape", ["auto", "block", "warps", "lowframe", "tight"])
 def test_allbroadcast_tables(forced_shape, shape, p, rank):
     forced_shape(shape)                                        # every launch shape of the table kernel
     orecv, osend = oracle.allbroadcast_schedule(p, rank)
@@ -298,7 +298,7 @@ def test_allbroadcast_large_p_is_the_reversed_broadcast_table(forced_shape):
     p, rank = workloads.P_MEDIUM, 777777
     recv0, send0 = bs.schedule(p)
     recv, send = bs.allbroadcast_schedule(p, rank)
-    for shape in ("warps", "block"):                       # the other shapes too (the deferred queue overflows here)
+    for shape in ("warps", "block", "tight"):              # the other shapes too (queues overflow in the last)
         forced_shape(shape)
         recv_w, send_w = bs.allbroadcast_schedule(p, rank)
         assert bool((recv_w == recv).all()) and bool((send_w == send).all()), shape
@@ -388,12 +388,13 @@ def test_table_kernel_against_batch_kernel_at_scale(p, root):
 
 
 # ------------------------------------------------------------------ both launch shapes of the table kernel
-@pytest.mark.parametrize("shape", ["block", "warps", "lowframe"])
+@pytest.mark.parametrize("shape", ["block", "warps", "lowframe", "tight"])
 @pytest.mark.parametrize("p,root", [(1000, 0), (5000, 1234), (2 ** 16 + 1, 7), (300007, 299999), (2 ** 20 + 1, 0),
                                     (2 ** 20 - 1, 5), (3 * 2 ** 18, 11), (999983, 500000)])
 def test_every_launch_shape_full_tables(forced_shape, shape, p, root):
     """The library picks the launch shape from an estimate; forced each way, on p with many and with few
-    undecided entries (the block's deferred queue overflows at p = 2^20 + 1), the tables equal the oracle's."""
+    undecided entries, the tables equal the oracle's.  The tight shape has next to no queue space, so every
+    group of tiles with undecided entries takes the path that recomputes its rows by the search alone."""
     forced_shape(shape)
     recv, send = gpu_tables(p, root)
     orecv, osend = oracle.schedule_table(p, root)
