@@ -321,13 +321,15 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     // up to kWarpsPerBlock consecutive tiles per block, fewer while the grid would have less than
     // kBlocksPerSmWanted blocks per SM (short launches want many small blocks).  A block that first
     // tabulates the search's low states takes more tiles to spread that cost: up to kLowFrameTiles,
-    // at least kWarpsPerBlock, aiming at four waves of resident blocks.
+    // aiming at four waves of resident blocks.
     int64_t tiles_per_block = n_tiles / ((int64_t)sms * kBlocksPerSmWanted);
     if (tiles_per_block < 1) tiles_per_block = 1;
     if (tiles_per_block > kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
     if (shape == kShapeWarpsLowFrame) {
         tiles_per_block = n_tiles / ((int64_t)sms * kTableBlocksPerSm * 4);
-        if (tiles_per_block < kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
+        // measured: 4 tiles at p = 2^20+1 (one wave of blocks), 8 at 2^22+1, 16-32 at 2^24+3, 64-128 at 1.2e8
+        const int least = n_tiles < (int64_t)sms * kTableBlocksPerSm * kWarpsPerBlock ? kWarpsPerBlock / 2 : kWarpsPerBlock;
+        if (tiles_per_block < least) tiles_per_block = least;
         if (tiles_per_block > kLowFrameTiles) tiles_per_block = kLowFrameTiles;
     }
     const int grid = (int)((n_tiles + tiles_per_block - 1) / tiles_per_block);
