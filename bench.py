@@ -55,7 +55,7 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as fh:
             return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+    return 6650.0, "fallback (6.65 TB/s: MEASURED_PEAKS.json is absent)"
 
 
 def kernel_source_hash() -> str:
@@ -69,20 +69,34 @@ def kernel_source_hash() -> str:
     return h.hexdigest()
 
 
-def recorded_traffic(kernel: str, p, filename: str = "dram_traffic.txt"):
-    """Sum of the two counters of one launch recorded in profiles/<filename> (DRAM bytes read + written, or
-    warp instructions + 0), or None when the sources changed since they were taken."""
-    path = os.path.join(ROOT, "profiles", filename)
+def recorded_counters(kernel: str, key: str):
+    """A line `kernel key sha256-of-csrc a b` of profiles/counters.txt as (a, b), or None when there is none for
+    the sources as they are now (ncu counters of a small stand-in launch; see the file for what a and b are)."""
+    path = os.path.join(ROOT, "profiles", "counters.txt")
     if not os.path.exists(path):
         return None
     sha = kernel_source_hash()
     with open(path) as fh:
         for line in fh:
             parts = line.split()
-            if len(parts) >= 5 and not line.startswith("#") and parts[0] == kernel and parts[1] == str(p) \
+            if len(parts) >= 5 and not line.startswith("#") and parts[0] == kernel and parts[1] == key \
                     and parts[2] == sha:
-                return int(parts[3]) + int(parts[4])
+                return float(parts[3]), float(parts[4])
     return None
+
+
+def scaled_traffic(kernel: str, key: str, algorithmic_bytes: float):
+    """DRAM bytes of one launch, scaled from the stand-in capture by the algorithmic bytes (a = DRAM bytes read +
+    written by the stand-in launch, b = its algorithmic bytes; the traffic is all table rows, so it grows with them)."""
+    rec = recorded_counters(kernel, key)
+    return None if rec is None else rec[0] / rec[1] * algorithmic_bytes
+
+
+def scaled_instructions(kernel: str, key: str, units: float):
+    """Warp instructions of one launch, scaled from the stand-in capture by the units processed (a = warp
+    instructions of the stand-in launch, b = its units)."""
+    rec = recorded_counters(kernel, key)
+    return None if rec is None else rec[0] / rec[1] * units
 
 
 def max_over_ranks(ms: float, world: int, device: str = "cuda") -> float:
@@ -186,6 +200,29 @@ def workload_label(mode: str, p: int, q: int, blocks: int = 0) -> str:
         return ("Algorithm 7 tables of processor %d for all roots of p=%d (q=%d), recvblocks+sendblocks int32"
                 % (p // 3, p, q))
     return "all ranks of p=%d (q=%d), root 0, recvblock+sendblock int32 tables" % (p, q)
+
+
+def oracle_other_modes(p: int):
+    """The oracle's other routes, timed beside the window mode (single thread, as it stands):
+    receive rows alone on a window of the same p, and the all-ranks route (receive rows by Algorithm 5 for
+    every rank, send rows gathered from them: one search per rank) on BASELINE config 2 in full."""
+    import oracle
+    from paper_2407_18004_b200 import workloads
+    rows = min(p, 2 ** 21)
+    t0 = time.perf_counter()
+    oracle.schedule_table(p, 0, 0, rows, want_send=False)
+    dt_recv = time.perf_counter() - t0
+    pm = workloads.P_MEDIUM
+    t0 = time.perf_counter()
+    oracle.schedule_table(pm, 0)
+    dt_all = time.perf_counter() - t0
+    return {
+        "recv_rows_only": {"value": rows / dt_recv, "unit": "rows/s", "seconds": dt_recv,
+                           "sample": "receive rows [0,%d) of p=%d by Algorithm 5 (one search per row)" % (rows, p)},
+        "all_ranks_mode": {"value": pm / dt_all, "unit": UNIT, "seconds": dt_all,
+                           "sample": "p=%d in full: receive rows by Algorithm 5, send rows gathered from them "
+                                     "(one search per rank)" % pm},
+    }
 
 
 def oracle_sample_size(p: int) -> int:
@@ -334,21 +371,31 @@ def run_ours(args):
         else:
             e2e = {"value": None, "unit": UNIT, "error": e2e_err}
 
+    peak, peak_src = measured_peaks()
+    store_only = None
+    configs = None
+    if world == 1 and args.mode == "broadcast":
+        store_only = measure_store_ceiling(bs, torch, recv, send, stream)
+        if not args.no_configs:
+            configs = measure_configs(bs, torch, recv, send, stream, peak, statistics.mean(per_step_ms), p)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return 0
 
-    peak, peak_src = measured_peaks()
     kernel_ms = statistics.mean(per_step_ms)
     achieved = table_bytes / (kernel_ms * 1e-3) / 1e9
-    traffic = recorded_traffic("schedule_table_kernel", p) if args.mode == "broadcast" else None
+    traffic = scaled_traffic("schedule_table_kernel", "clean", table_bytes) if args.mode == "broadcast" else None
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         v, dt, sample = time_oracle_sample(p, oracle_sample_size(p), args.mode, args.blocks)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-                        "seconds": dt, "host_cores_available": os.cpu_count()}
+                        "seconds": dt, "host_cores_available": os.cpu_count(),
+                        "mode": "window (q + 1 searches per rank: the oracle's slowest route)"}
+        if args.mode == "broadcast":
+            cpu_baseline.update(oracle_other_modes(p))
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -363,16 +410,136 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "kernel": "schedule_table_kernel", "bytes_per_launch": table_bytes,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "store_only_gbs": store_only,
+                     "frac_of_store_only": achieved / store_only if store_only else None},
         "cpu_baseline": cpu_baseline,
         "e2e": e2e,
         "gpu_launches": args.steps,
         "clocks": clocks,
     }
+    if configs is not None:
+        line["configs"] = configs
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def time_launches(torch, stream, fn, pairs: int, per_pair: int = 1, before=None):
+    """Mean and minimum device time in ms of one call of fn: `pairs` event pairs, each around `per_pair` calls
+    back to back (short launches are timed many to a pair)."""
+    times = []
+    for _ in range(pairs):
+        if before is not None:
+            before()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(per_pair):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / per_pair)
+    return statistics.mean(times), min(times)
+
+
+def measure_store_ceiling(bs, torch, recv, send, stream):
+    """GB/s of bcast_store_ceiling over the same bytes as the headline tables (both buffers, one launch each)."""
+    def fill():
+        bs.bcast_store_ceiling(recv, recv.numel() * 4, 0, stream)
+        bs.bcast_store_ceiling(send, send.numel() * 4, 0, stream)
+    fill()
+    torch.cuda.synchronize()
+    mean_ms, _ = time_launches(torch, stream, fill, 5)
+    return (recv.numel() + send.numel()) * 4 / (mean_ms * 1e-3) / 1e9
+
+
+def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
+    """The other BASELINE configurations and the library's other table forms, measured in the same run (same
+    device buffers, same clock sampling window is not repeated: short runs).  Each entry: mean ms per launch, the
+    workload's own throughput, and the roofline fraction with its bound."""
+    from paper_2407_18004_b200 import workloads
+    flat_r, flat_s = recv.view(-1), send.view(-1)
+    out = {}
+
+    def tables(p):
+        q = bs.bcast_q(p)
+        return q, flat_r[:p * q].view(p, q), flat_s[:p * q].view(p, q)
+
+    def table_entry(name, p, launch, pairs, per_pair, what):
+        q, r, s_ = tables(p)
+        fn = lambda: launch(p, q, r, s_)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        mean_ms, min_ms = time_launches(torch, stream, fn, pairs, per_pair)
+        nbytes = 8 * q * p
+        gbs = nbytes / (mean_ms * 1e-3) / 1e9
+        out[name] = {"workload": what % (p, q), "ms": mean_ms, "ms_min": min_ms, "launches_per_event_pair": per_pair,
+                     "value": p / (mean_ms * 1e-3), "unit": UNIT, "bytes_per_launch": nbytes,
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak}}
+        return mean_ms
+
+    table_entry("config2_p=2^20+1", workloads.P_MEDIUM,
+                lambda p, q, r, s_: bs.bcast_schedule(p, 0, 0, p, r, s_, stream), 5, 60,
+                "all ranks of p=%d (q=%d), root 0 (BASELINE config 2); tables larger than L2, launches back to back")
+    table_entry("ordinary_p=123456789", 123456789,
+                lambda p, q, r, s_: bs.bcast_schedule(p, 0, 0, p, r, s_, stream), 10, 1,
+                "all ranks of p=%d (q=%d), root 0: a p with no special form")
+    ms_root = table_entry("root_p/3_p=2^27-1", p_large,
+                          lambda p, q, r, s_: bs.bcast_schedule(p, p // 3, 0, p, r, s_, stream), 10, 1,
+                          "all ranks of p=%d (q=%d), root floor(p/3)")
+    out["root_p/3_p=2^27-1"]["ms_over_root_0"] = ms_root / headline_ms
+    table_entry("allbroadcast_p=2^27-1", p_large,
+                lambda p, q, r, s_: bs.bcast_allbroadcast_schedule(p, p // 3, 0, p, r, s_, stream), 10, 1,
+                "Algorithm 7's tables of processor floor(p/3) for all roots of p=%d (q=%d)")
+    table_entry("shifted_n=64_p=2^27-1", p_large,
+                lambda p, q, r, s_: bs.bcast_schedule_shifted(p, 0, 64, 0, p, r, s_, stream), 10, 1,
+                "all ranks of p=%d (q=%d), root 0, rows after Algorithm 1's preamble for n=64 blocks")
+
+    # config 5: 2^24 independent queries (rows padded to 31), outputs in the same buffers
+    nq = 2 ** 24
+    hp, hr, ho = workloads.query_batch(nq, seed=0)
+    dp, dr, do = [torch.from_numpy(a).cuda() for a in (hp, hr, ho)]
+    brecv, bsend = flat_r[:nq * 31].view(nq, 31), flat_s[:nq * 31].view(nq, 31)
+    bad = torch.zeros(1, dtype=torch.int32, device="cuda")
+    batch = lambda: bs.bcast_schedule_batch(dp, dr, do, 31, brecv, bsend, bad, stream)
+    for _ in range(3):
+        batch()
+    torch.cuda.synchronize()
+    mean_ms, min_ms = time_launches(torch, stream, batch, 10)
+    insts = scaled_instructions("schedule_batch_kernel", "batch", nq)
+    ach = insts / (mean_ms * 1e-3) / 1e9 if insts else None
+    out["config5_batch_2^24"] = {
+        "workload": "2^24 queries, p log-uniform in [2, 2^31-1], rank and root uniform, seed 0, rows padded to 31 "
+                    "(BASELINE config 5)", "ms": mean_ms, "ms_min": min_ms, "value": nq / (mean_ms * 1e-3),
+        "unit": "queries/s", "bytes_per_launch": nq * (2 * 31 * 4 + 12),
+        "hbm_write_gbs": nq * 2 * 31 * 4 / (mean_ms * 1e-3) / 1e9,
+        "roofline": {"bound": "alu", "achieved": ach, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
+                     "frac": ach / ISSUE_PEAK_GINST if ach else None, "warp_instructions_per_launch": insts}}
+    del dp, dr, do
+
+    # config 4: the fused verification sweep
+    lo, hi = 2, 65536
+    checksum = torch.zeros(hi - lo + 1, dtype=torch.int64, device="cuda")
+    fails = torch.zeros(8, dtype=torch.int32, device="cuda")
+    need = bs.bcast_verify_sweep_scratch_bytes(lo, hi)
+    scratch = flat_r.view(torch.uint8)[:need]
+    sweep = lambda: bs.bcast_verify_sweep(lo, hi, checksum, fails, scratch, stream)
+    sweep()
+    torch.cuda.synchronize()
+    mean_ms, min_ms = time_launches(torch, stream, sweep, 3)
+    units = sum(range(lo, hi + 1))
+    insts = scaled_instructions("verify_sweep_kernel", "sweep", units)
+    ach = insts / (mean_ms * 1e-3) / 1e9 if insts else None
+    out["config4_sweep_2_65536"] = {
+        "workload": "every p in [2, 65536], all ranks, root 0: tables built and checked on the device, one checksum "
+                    "per p (BASELINE config 4)", "ms": mean_ms, "ms_min": min_ms, "value": units / (mean_ms * 1e-3),
+        "unit": "rank-schedules/s", "fail_counts": fails.tolist(),
+        "roofline": {"bound": "alu", "achieved": ach, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
+                     "frac": ach / ISSUE_PEAK_GINST if ach else None, "warp_instructions_per_launch": insts}}
+    return out
 
 
 # ---------------------------------------------------------------------------------------------
@@ -609,13 +776,13 @@ def run_other(args):
         peak, peak_src = measured_peaks()
         achieved = wl["bytes"] / (mean_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": recorded_traffic(wl["kernel"], args.mode), "peak_source": peak_src,
+                    "traffic": None, "peak_source": peak_src,
                     "kernel": wl["kernel"], "bytes_per_step": wl["bytes"],
                     "note": "algorithmic bytes of the whole step over the step's time (many short launches)"}
     else:
         # bound by instruction issue: warp instructions of one launch (recorded from ncu while the sources
         # are unchanged) over its time, against one instruction per scheduler and clock
-        insts = recorded_traffic(wl["kernel"], args.mode, "warp_instructions.txt")
+        insts = scaled_instructions(wl["kernel"], args.mode, wl["units"])
         achieved = insts / (mean_ms * 1e-3) / 1e9 if insts else None
         roofline = {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
                     "frac": achieved / ISSUE_PEAK_GINST if achieved else None, "traffic": None,
@@ -738,6 +905,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the other BASELINE configurations that the default run measures beside the headline")
     args = ap.parse_args()
     if args.mode in OTHER_MODES:
         if args.workload == "p=2^27-1":

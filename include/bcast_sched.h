@@ -316,6 +316,17 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
                           void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
 
 /*
+ * Measurement aid (no counterpart in the paper): fills buffer_dev (device,
+ * 16-byte aligned; bytes rounded down to a multiple of 16) with the store
+ * pattern of the table kernel and nothing else -- one block of 256 threads per
+ * contiguous chunk of bytes_per_block bytes (0: the bytes a block of
+ * bcast_schedule writes at q = 27), 16-byte streaming stores.  Its rate is the
+ * write-only ceiling the table kernel's HBM fraction can be read against.
+ * Asynchronous on cuda_stream.  Returns BCAST_OK or a BCAST_E* code.
+ */
+int bcast_store_ceiling(void *buffer_dev, int64_t bytes, int64_t bytes_per_block, void *cuda_stream);
+
+/*
  * Algorithm 1's use of a schedule row, O(1) per round.  For n >= 1 blocks and
  * communication round j in [0, n-1+q): x = (q - (n-1) mod q) mod q virtual
  * rounds come first, so i = x + j, k = i mod q is the skip index of the round

@@ -61,6 +61,8 @@ def _load():
             lib.oracle_checksum.argtypes = [i64, u64p]
             lib.oracle_schedule_batch.argtypes = [i32p, i32p, i32p, i64, ctypes.c_int32,
                                                   ctypes.c_int32, i32p, i32p]
+            lib.oracle_sendschedule_alg6_batch.argtypes = [i32p, i32p, i32p, i64, ctypes.c_int32,
+                                                           ctypes.c_int32, i32p]
             lib.oracle_shift_rows.argtypes = [ctypes.c_int, i64, i64, i32p]
             lib.oracle_simulate_broadcast.argtypes = [i64, i64, i64, i32p, i32p, i32p, u64p]
             lib.oracle_simulate_reduce.argtypes = [i64, i64, i64, i32p, i32p, u64p, u64p, u64p]
@@ -218,6 +220,18 @@ def schedule_batch(p, rank, root, row_stride: int = 31, pad: int = PAD,
     if rc < 0:
         raise ValueError("bad query in batch")
     return recv, send
+
+
+def sendschedule_alg6_batch(p, rank, root, row_stride: int = 31, pad: int = PAD) -> np.ndarray:
+    """Send rows of independent queries by Algorithm 6 (second routine), padded to row_stride."""
+    p = np.ascontiguousarray(p, dtype=np.int32)
+    rank = np.ascontiguousarray(rank, dtype=np.int32)
+    root = np.ascontiguousarray(root, dtype=np.int32)
+    nq = p.shape[0]
+    send = np.zeros((nq, row_stride), dtype=np.int32)
+    if _load().oracle_sendschedule_alg6_batch(_i32(p), _i32(rank), _i32(root), nq, row_stride, pad, _i32(send)) < 0:
+        raise ValueError("bad query in batch")
+    return send
 
 
 def _u64(a):

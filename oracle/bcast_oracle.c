@@ -503,6 +503,28 @@ int oracle_schedule_batch(const int32_t *p, const int32_t *rank, const int32_t *
 }
 
 /*
+ * Send rows of independent queries by Algorithm 6 (the second routine, see
+ * oracle_sendschedule_alg6), padded like oracle_schedule_batch.  The tests use
+ * it where q receive schedules per query (the definition) would take too long.
+ */
+int oracle_sendschedule_alg6_batch(const int32_t *p, const int32_t *rank, const int32_t *root,
+                                   int64_t nq, int32_t row_stride, int32_t pad, int32_t *send_out)
+{
+    int64_t i;
+    int k;
+    for (i = 0; i < nq; i++) {
+        int64_t pi = p[i], r;
+        int q = oracle_q(pi);
+        if (q < 0 || q > row_stride || rank[i] < 0 || rank[i] >= pi || root[i] < 0 || root[i] >= pi)
+            return -1;
+        r = ((int64_t)rank[i] - root[i] + pi) % pi;
+        if (oracle_sendschedule_alg6(pi, r, send_out + i * row_stride, NULL, NULL) < 0) return -1;
+        for (k = q; k < row_stride; k++) send_out[i * row_stride + k] = pad;
+    }
+    return 0;
+}
+
+/*
  * Algorithm 1's preamble for a whole table: the rows Broadcast() starts its
  * communication loop with when n blocks are broadcast.  With
  * x = (q - (n-1) mod q) mod q every entry has x subtracted, and the entries of

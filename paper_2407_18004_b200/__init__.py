@@ -54,6 +54,7 @@ def _load():
         lib.bcast_simulate_scratch_bytes.restype = i64
         lib.bcast_simulate_broadcast.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_simulate_reduce.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, vp, i64, vp]
+        lib.bcast_store_ceiling.argtypes = [vp, i64, i64, vp]
         lib.bcast_round.argtypes = [i32, i64, i64, ctypes.POINTER(i32), ctypes.POINTER(i64)]
         lib.bcast_round_block.argtypes = [i32, i64, i64, vp]
         lib.bcast_round_block.restype = i64
@@ -106,6 +107,10 @@ def bcast_skips(p: int) -> np.ndarray:
     out = np.zeros(q + 1, dtype=np.int32)
     _check(_load().bcast_skips(p, out.ctypes.data))
     return out
+
+
+def bcast_store_ceiling(buffer, nbytes: int, bytes_per_block: int = 0, stream=None) -> int:
+    return _check(_load().bcast_store_ceiling(_ptr(buffer), nbytes, bytes_per_block, _stream(stream)))
 
 
 def bcast_round(q: int, n: int, j: int):

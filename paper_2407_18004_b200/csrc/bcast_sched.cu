@@ -182,6 +182,18 @@ schedule_batch_kernel(const int32_t *__restrict__ p_in, const int32_t *__restric
     }
 }
 
+// ------------------------------------------------------------------ write-only ceiling
+// Nothing but the table kernel's store pattern: every block streams out one contiguous chunk
+// with 16-byte st.global.cs, a warp covering 512 contiguous bytes per instruction.
+__global__ void __launch_bounds__(kThreads)
+store_ceiling_kernel(int4 *__restrict__ out, int64_t n_vec, int64_t vec_per_block)
+{
+    const int64_t begin = (int64_t)blockIdx.x * vec_per_block;
+    const int64_t end = min(begin + vec_per_block, n_vec);
+    const int4 v = make_int4((int)blockIdx.x, (int)threadIdx.x, -1, -2);
+    for (int64_t i = begin + threadIdx.x; i < end; i += kThreads) __stcs(out + i, v);
+}
+
 }  // namespace bcast
 
 using namespace bcast;
@@ -470,6 +482,23 @@ int bcast_schedule_batch(const int32_t *p_dev, const int32_t *rank_dev, const in
     schedule_batch_kernel<<<grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
         p_dev, rank_dev, root_dev, nq, row_stride, recvblock_dev, sendblock_dev, bad_count_dev,
         ((uintptr_t)recvblock_dev & 15u) == 0, ((uintptr_t)sendblock_dev & 15u) == 0);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return BCAST_OK;
+}
+
+int bcast_store_ceiling(void *buffer_dev, int64_t bytes, int64_t bytes_per_block, void *cuda_stream)
+{
+    if (buffer_dev == nullptr) return BCAST_ENULL;
+    if ((uintptr_t)buffer_dev & 15u) return BCAST_EALIGN;
+    if (bytes < 0 || bytes_per_block < 0) return BCAST_EINVAL_N;
+    if (bytes_per_block == 0) bytes_per_block = (int64_t)kWarpsPerBlock * kThreads * 27 * 8;   // 8 tiles of both tables at q = 27
+    const int64_t n_vec = bytes / 16;
+    const int64_t vec_per_block = (bytes_per_block + 15) / 16;
+    if (n_vec == 0) return BCAST_OK;
+    const int64_t grid = (n_vec + vec_per_block - 1) / vec_per_block;
+    if (grid > 0x7fffffff) return BCAST_EINVAL_N;
+    store_ceiling_kernel<<<(int)grid, kThreads, 0, (cudaStream_t)cuda_stream>>>(
+        reinterpret_cast<int4 *>(buffer_dev), n_vec, vec_per_block);
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return BCAST_OK;
 }

@@ -2,16 +2,24 @@
 path has no exchange step): rank 0 alone prints the JSON line, the other rank exits 0 silently."""
 import json
 import os
+import socket
 import subprocess
 import sys
 
 from conftest import ROOT
 
 
+def free_port() -> str:
+    """A TCP port nobody listens on right now (two test runs side by side must not meet on a fixed one)."""
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return str(sock.getsockname()[1])
+
+
 def test_reference_arm_two_processes():
     env = dict(os.environ, MASTER_ADDR="127.0.0.1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29731", os.path.join(ROOT, "bench.py"),
+           "--master-addr", "127.0.0.1", "--master-port", free_port(), os.path.join(ROOT, "bench.py"),
            "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--workload", "p=1000"]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
@@ -50,7 +58,7 @@ def test_max_over_ranks_and_whole_job_value_two_gloo_ranks():
     # the replicas of a multi-GPU run are timed as the slowest rank and counted together
     env = dict(os.environ, MASTER_ADDR="127.0.0.1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29733", os.path.join(ROOT, "tests", "dist_worker.py")]
+           "--master-addr", "127.0.0.1", "--master-port", free_port(), os.path.join(ROOT, "tests", "dist_worker.py")]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [l for l in out.stdout.splitlines() if l.startswith("{")]

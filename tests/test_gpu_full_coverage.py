@@ -1,0 +1,106 @@
+"""Full-coverage parity at the benchmark's sizes (-m gpu), against the CPU oracle alone.
+
+The oracle is single-threaded; these tests run it in a pool of processes (one per host core, at most
+16, started with spawn) on chunks of the workload while the device rows of each chunk are brought
+back as int8 and compared element by element.
+
+  config 3  every receive row of p = 2^27-1 (134 217 727 rows; about two minutes of one core), and then
+            condition 2 over the whole device tables, which with a verified receive table IS the
+            definition of the send table (Section 2.3);
+  config 4  the checksum of every p in [2, 65536] against tests/golden/checksums_2_65536.txt, which
+            tests/golden/make_checksums.py wrote from the oracle;
+  config 5  every receive row of the 2^24 queries against Algorithm 5 and every send row against the
+            oracle's Algorithm 6 routine (about a minute of one core), plus the definition of the send
+            row (q receive schedules per query) on a sample.
+"""
+import multiprocessing as mp
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import oracle_workers
+import paper_2407_18004_b200 as bs
+from conftest import GOLDEN
+from paper_2407_18004_b200 import workloads
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def first_difference(name, got, want, lo):
+    if got.shape != want.shape:
+        return "%s: shape %s vs %s" % (name, got.shape, want.shape)
+    bad = np.argwhere(got != want)
+    if len(bad) == 0:
+        return None
+    r, k = bad[0]
+    return "%s: %d entries differ, first at row %d round %d: device %d, oracle %d" % (
+        name, len(bad), lo + r, k, got[r, k], want[r, k])
+
+
+def test_config3_every_receive_row_and_the_send_table_by_definition():
+    p = workloads.P_LARGE
+    q = bs.bcast_q(p)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 34 * 2 ** 30:
+        pytest.skip("needs 34 GB of device memory")
+    oracle.build()
+    recv, send = bs.schedule(p)
+    torch.cuda.synchronize()
+    chunk = 2 ** 22
+    jobs = [(p, 0, lo, min(p, lo + chunk)) for lo in range(0, p, chunk)]
+    with mp.get_context("spawn").Pool(oracle_workers.pool_size()) as pool:
+        for (_, _, lo, hi), want in zip(jobs, pool.imap(oracle_workers.recv_rows, jobs)):
+            got = recv[lo:hi].to(torch.int8).cpu().numpy()
+            msg = first_difference("recvblock", got, want, lo)
+            assert msg is None, msg
+    # Section 2.3: sendblock[k] of r is recvblock[k] of (r + skip[k]) mod p, for every rank and round
+    skips = bs.bcast_skips(p)
+    ranks = torch.arange(p, device="cuda")
+    for k in range(q):
+        to = (ranks + int(skips[k])) % p
+        assert bool((send[:, k] == recv[to, k]).all()), "send table differs from its definition in round %d" % k
+        del to
+
+
+def test_config4_every_checksum_against_the_golden_file():
+    with open(os.path.join(GOLDEN, "checksums_2_65536.txt")) as fh:
+        want = np.array([int(line, 16) for line in fh if not line.startswith("#")], dtype=np.uint64)
+    assert want.shape == (65535,)
+    checksum, fails = bs.verify_sweep(2, 65536)
+    torch.cuda.synchronize()
+    assert fails.tolist() == [0] * 8
+    got = checksum.cpu().numpy().view(np.uint64)
+    bad = np.nonzero(got != want)[0]
+    assert len(bad) == 0, "checksums differ for %d values of p, first p = %d" % (len(bad), bad[0] + 2)
+
+
+def test_config5_every_query_row():
+    nq = 2 ** 24
+    free, _ = torch.cuda.mem_get_info()
+    if free < 6 * 2 ** 30:
+        pytest.skip("needs 6 GB of device memory")
+    oracle.build()
+    hp, hr, ho = workloads.query_batch(nq, seed=0)
+    recv, send, bad = bs.schedule_batch(torch.from_numpy(hp).cuda(), torch.from_numpy(hr).cuda(),
+                                        torch.from_numpy(ho).cuda(), 31)
+    torch.cuda.synchronize()
+    assert int(bad) == 0
+    chunk = 2 ** 19
+    bounds = [(lo, min(nq, lo + chunk)) for lo in range(0, nq, chunk)]
+    jobs = [(hp[lo:hi], hr[lo:hi], ho[lo:hi]) for lo, hi in bounds]
+    with mp.get_context("spawn").Pool(oracle_workers.pool_size()) as pool:
+        for (lo, hi), (want_r, want_s) in zip(bounds, pool.imap(oracle_workers.batch_rows, jobs)):
+            got_r = recv[lo:hi].clamp(min=-128).to(torch.int8).cpu().numpy()     # BCAST_PAD -> -128
+            got_s = send[lo:hi].clamp(min=-128).to(torch.int8).cpu().numpy()
+            msg = first_difference("recv rows", got_r, want_r, lo) or first_difference("send rows (Algorithm 6)",
+                                                                                       got_s, want_s, lo)
+            assert msg is None, msg
+    # the send row by its definition, q receive schedules per query, on a sample spread over the batch
+    idx = np.arange(0, nq, nq // 2 ** 15)
+    _, want = oracle.schedule_batch(hp[idx], hr[idx], ho[idx], 31, bs.BCAST_PAD, want_recv=False)
+    got = send[torch.from_numpy(idx).cuda()].cpu().numpy()
+    msg = first_difference("send rows (definition)", got, want, 0)
+    assert msg is None, msg
