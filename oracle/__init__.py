@@ -66,6 +66,8 @@ def _load():
             lib.oracle_shift_rows.argtypes = [ctypes.c_int, i64, i64, i32p]
             lib.oracle_simulate_broadcast.argtypes = [i64, i64, i64, i32p, i32p, i32p, u64p]
             lib.oracle_simulate_reduce.argtypes = [i64, i64, i64, i32p, i32p, u64p, u64p, u64p]
+            lib.oracle_simulate_allbroadcast.argtypes = [i64, i64, i32p, i32p, i32p, u64p]
+            lib.oracle_simulate_allreduce.argtypes = [i64, i64, i32p, i32p, u64p, u64p, u64p]
             _lib = lib
     return _lib
 
@@ -278,4 +280,40 @@ def simulate_reduce(p: int, root: int, n: int, recv_tab, send_tab, value):
     if _load().oracle_simulate_reduce(p, root, n, _i32(recv_tab), _i32(send_tab), _u64(work), _u64(result),
                                       _u64(stats)) < 0:
         raise ValueError("bad arguments to simulate_reduce")
+    return result, stats
+
+
+def simulate_allbroadcast(p: int, n: int, recv0=None, send0=None):
+    """Algorithm 7 by all processors: (arrival[p roots][n][p] int32, stats[8] uint64).
+
+    recv0/send0 None: every processor's tables by Algorithm 7's own loops; else the root-0 broadcast
+    tables [p][q] whose row (r - j) mod p serves processor r for root j (for damaged tables).
+    """
+    q = q_of(p)
+    given = recv0 is not None and send0 is not None
+    if given:
+        recv0 = np.ascontiguousarray(recv0, dtype=np.int32).reshape(p, q)
+        send0 = np.ascontiguousarray(send0, dtype=np.int32).reshape(p, q)
+    arrival = np.zeros((p, n, p), dtype=np.int32)
+    stats = np.zeros(8, dtype=np.uint64)
+    if _load().oracle_simulate_allbroadcast(p, n, _i32(recv0) if given else None, _i32(send0) if given else None,
+                                            _i32(arrival), _u64(stats)) < 0:
+        raise ValueError("bad arguments to simulate_allbroadcast")
+    return arrival, stats
+
+
+def simulate_allreduce(p: int, n: int, value, recv0=None, send0=None):
+    """Observation 1.4's all-reduction (wrapping 64-bit sum): value [p roots][n][p] uint64 contributions
+    (not modified).  Returns (result[p][n] uint64, stats[8] uint64).  Tables as for simulate_allbroadcast."""
+    q = q_of(p)
+    given = recv0 is not None and send0 is not None
+    if given:
+        recv0 = np.ascontiguousarray(recv0, dtype=np.int32).reshape(p, q)
+        send0 = np.ascontiguousarray(send0, dtype=np.int32).reshape(p, q)
+    work = np.array(value, dtype=np.uint64, copy=True).reshape(p, n, p)
+    result = np.zeros((p, n), dtype=np.uint64)
+    stats = np.zeros(8, dtype=np.uint64)
+    if _load().oracle_simulate_allreduce(p, n, _i32(recv0) if given else None, _i32(send0) if given else None,
+                                         _u64(work), _u64(result), _u64(stats)) < 0:
+        raise ValueError("bad arguments to simulate_allreduce")
     return result, stats

@@ -750,3 +750,234 @@ int oracle_simulate_reduce(int64_t p, int64_t root, int64_t n,
     free(wire); free(wire_val); free(times_sent);
     return q;
 }
+
+/*
+ * Tables of Algorithm 7 for every processor: recvs[r][j][k], sends[r][j][k] for
+ * processor r and root j.  With recv0/send0 == NULL they come from
+ * oracle_allbroadcast_schedule, processor by processor, as the algorithm prints
+ * them.  Otherwise processor r's row for root j is row (r - j) mod p of the
+ * given root-0 broadcast tables (which is what the printed loops amount to; the
+ * tests pin that equality), so that damaged tables can be tried.
+ */
+static int all_tables_(int64_t p, int q, const int32_t *recv0, const int32_t *send0,
+                       int32_t **recvs_out, int32_t **sends_out)
+{
+    int64_t r, j;
+    int k;
+    size_t cells = (size_t)p * (size_t)p * (size_t)q;
+    int32_t *recvs = (int32_t *)malloc(cells * sizeof(int32_t) + 1);
+    int32_t *sends = (int32_t *)malloc(cells * sizeof(int32_t) + 1);
+    if (!recvs || !sends) { free(recvs); free(sends); return -2; }
+    for (r = 0; r < p; r++) {
+        if (recv0 == NULL || send0 == NULL) {
+            if (oracle_allbroadcast_schedule(p, r, 0, p, recvs + (size_t)r * p * q, sends + (size_t)r * p * q) < 0) {
+                free(recvs); free(sends); return -1;
+            }
+        } else {
+            for (j = 0; j < p; j++) {
+                int64_t v = (r - j + p) % p;
+                for (k = 0; k < q; k++) {
+                    recvs[((size_t)r * p + j) * q + k] = recv0[v * q + k];
+                    sends[((size_t)r * p + j) * q + k] = send0[v * q + k];
+                }
+            }
+        }
+    }
+    *recvs_out = recvs;
+    *sends_out = sends;
+    return 0;
+}
+
+/* Block of a table entry in round i: Algorithm 7's shift by -x, one q per phase; -1: nothing. */
+static int64_t round_block_(int32_t entry, int q, int64_t i, int64_t x, int64_t n)
+{
+    int64_t blk;
+    if (entry < -q || entry > q - 1) return -1;
+    blk = (int64_t)entry + (i / q) * q - x;
+    if (blk < 0) return -1;
+    return blk > n - 1 ? n - 1 : blk;
+}
+
+/*
+ * Algorithm 7 run by all p processors in lock-step: every processor is the root
+ * of a broadcast of its own n blocks, all p broadcasts share the rounds.  In
+ * round i (k = i mod q) processor r packs, for every root j but its
+ * to-processor t = (r + skip[k]) mod p, block sendblocks[j][k]; after the
+ * exchange it unpacks, for every root j but itself, block recvblocks[j][k] from
+ * what its from-processor f = (r - skip[k]) mod p packed for root j.  Negative
+ * blocks are not packed or unpacked, a block above n-1 stands for n-1.
+ *
+ * arrival[(j * n + b) * p + r]: the round (from 1) in which processor r got
+ * block b of root j; 0 for r = j; -1 if never.  A block is delivered only if
+ * the sender packed exactly the block the receiver unpacks for that root, held
+ * it before the round, and the receiver does not hold it yet.
+ * stats[0..7] as for oracle_simulate_broadcast, summed over all roots.
+ */
+int oracle_simulate_allbroadcast(int64_t p, int64_t n, const int32_t *recv0, const int32_t *send0,
+                                 int32_t *arrival, uint64_t *stats)
+{
+    int q = oracle_q(p);
+    int64_t skip[ORACLE_MAXQ + 2];
+    int64_t x, i, r, j, b;
+    int32_t *recvs = NULL, *sends = NULL;
+    int64_t *wire;
+    unsigned char *wire_held;
+    int k, rc;
+    if (q < 0 || n < 1) return -1;
+    memset(stats, 0, 8 * sizeof(uint64_t));
+    for (j = 0; j < p; j++)
+        for (b = 0; b < n; b++)
+            for (r = 0; r < p; r++) arrival[(j * n + b) * p + r] = (r == j) ? 0 : -1;
+    if (q == 0) return 0;
+    oracle_skips(p, skip);
+    rc = all_tables_(p, q, recv0, send0, &recvs, &sends);
+    if (rc < 0) return rc;
+    wire = (int64_t *)malloc((size_t)p * p * sizeof(int64_t));
+    wire_held = (unsigned char *)malloc((size_t)p * p);
+    if (!wire || !wire_held) { free(recvs); free(sends); free(wire); free(wire_held); return -2; }
+    for (r = 0; r < p; r++)
+        for (j = 0; j < p; j++)
+            for (k = 0; k < q; k++) {
+                int32_t rv = recvs[((size_t)r * p + j) * q + k], sv = sends[((size_t)r * p + j) * q + k];
+                if (rv < -q || rv > q - 1) stats[5]++;
+                if (sv < -q || sv > q - 1) stats[5]++;
+            }
+    x = (q - (n - 1) % q) % q;
+    for (i = x; i < n + q - 1 + x; i++) {
+        int64_t round = i - x + 1;
+        k = (int)(i % q);
+        /* pack: from what every processor held before the round */
+        for (r = 0; r < p; r++) {
+            int64_t t = (r + skip[k]) % p;
+            for (j = 0; j < p; j++) {
+                int64_t blk = -1;
+                if (j != t) blk = round_block_(sends[((size_t)r * p + j) * q + k], q, i, x, n);
+                wire[r * p + j] = blk;
+                wire_held[r * p + j] = (blk >= 0 && arrival[(j * n + blk) * p + r] >= 0);
+            }
+        }
+        /* unpack */
+        for (r = 0; r < p; r++) {
+            int64_t f = (r - skip[k] + p) % p;
+            for (j = 0; j < p; j++) {
+                int64_t want;
+                if (j == r) continue;
+                want = round_block_(recvs[((size_t)r * p + j) * q + k], q, i, x, n);
+                if (want < 0) {
+                    if (wire[f * p + j] >= 0) stats[3]++;
+                } else if (wire[f * p + j] != want) {
+                    stats[0]++;
+                } else if (!wire_held[f * p + j]) {
+                    stats[1]++;
+                } else if (arrival[(j * n + want) * p + r] >= 0) {
+                    stats[2]++;
+                } else {
+                    arrival[(j * n + want) * p + r] = (int32_t)round;
+                    stats[6]++;
+                    stats[7] = (uint64_t)round;
+                }
+            }
+        }
+    }
+    for (j = 0; j < p; j++)
+        for (b = 0; b < n; b++)
+            for (r = 0; r < p; r++)
+                if (arrival[(j * n + b) * p + r] < 0) stats[4]++;
+    free(recvs); free(sends); free(wire); free(wire_held);
+    return q;
+}
+
+/*
+ * The all-reduction of Observation 1 (item 4): Algorithm 7's rounds taken from
+ * the last to the first with every communication reversed, all p reductions
+ * sharing the rounds.  In the round that is all-broadcast round i, processor r
+ * packs, for every root j but itself, its partial result of block
+ * recvblocks[j][k] and sends the message to its from-processor f; from its
+ * to-processor t it receives, for every root j but t, a partial result of block
+ * sendblocks[j][k], which it adds to its own.  Negative blocks move nothing, a
+ * block above n-1 stands for n-1.
+ *
+ * value[(j * n + b) * p + r]: processor r's contribution to block b of root j
+ * (overwritten with partial results); the operator is the wrapping 64-bit sum.
+ * result[j * n + b]: root j's value of its block b after the last round, the
+ * sum over all processors for correct tables.  A partial result is combined
+ * only if the receiver expects exactly the block the sender packed for that
+ * root and has not passed (and is not passing) its own partial result of it on.
+ * stats[0..7] as for oracle_simulate_reduce, summed over all roots.
+ */
+int oracle_simulate_allreduce(int64_t p, int64_t n, const int32_t *recv0, const int32_t *send0,
+                              uint64_t *value, uint64_t *result, uint64_t *stats)
+{
+    int q = oracle_q(p);
+    int64_t skip[ORACLE_MAXQ + 2];
+    int64_t x, i, r, j, b;
+    int32_t *recvs = NULL, *sends = NULL;
+    int64_t *wire;
+    uint64_t *wire_val;
+    int32_t *times_sent;
+    int k, rc;
+    if (q < 0 || n < 1) return -1;
+    memset(stats, 0, 8 * sizeof(uint64_t));
+    if (q == 0) { for (b = 0; b < n; b++) result[b] = value[b]; return 0; }
+    oracle_skips(p, skip);
+    rc = all_tables_(p, q, recv0, send0, &recvs, &sends);
+    if (rc < 0) return rc;
+    wire = (int64_t *)malloc((size_t)p * p * sizeof(int64_t));
+    wire_val = (uint64_t *)malloc((size_t)p * p * sizeof(uint64_t));
+    times_sent = (int32_t *)calloc((size_t)p * p * n, sizeof(int32_t));
+    if (!wire || !wire_val || !times_sent) {
+        free(recvs); free(sends); free(wire); free(wire_val); free(times_sent);
+        return -2;
+    }
+    for (r = 0; r < p; r++)
+        for (j = 0; j < p; j++)
+            for (k = 0; k < q; k++) {
+                int32_t rv = recvs[((size_t)r * p + j) * q + k], sv = sends[((size_t)r * p + j) * q + k];
+                if (rv < -q || rv > q - 1) stats[5]++;
+                if (sv < -q || sv > q - 1) stats[5]++;
+            }
+    x = (q - (n - 1) % q) % q;
+    for (i = n + q - 1 + x - 1; i >= x; i--) {
+        k = (int)(i % q);
+        /* pack: every processor's partial results as they are before the round */
+        for (r = 0; r < p; r++)
+            for (j = 0; j < p; j++) {
+                int64_t blk = -1;
+                if (j != r) blk = round_block_(recvs[((size_t)r * p + j) * q + k], q, i, x, n);
+                wire[r * p + j] = blk;
+                if (blk >= 0) {
+                    wire_val[r * p + j] = value[(j * n + blk) * p + r];
+                    if (times_sent[(j * n + blk) * p + r] > 0) stats[2]++;
+                }
+            }
+        /* unpack and combine */
+        for (r = 0; r < p; r++) {
+            int64_t t = (r + skip[k]) % p;
+            for (j = 0; j < p; j++) {
+                int64_t want = -1;
+                if (j != t) want = round_block_(sends[((size_t)r * p + j) * q + k], q, i, x, n);
+                if (want < 0) {
+                    if (j != t && wire[t * p + j] >= 0) stats[3]++;
+                } else if (wire[t * p + j] != want) {
+                    stats[0]++;
+                } else if (r != j && (times_sent[(j * n + want) * p + r] > 0 || wire[r * p + j] == want)) {
+                    stats[1]++;
+                } else {
+                    value[(j * n + want) * p + r] += wire_val[t * p + j];
+                    stats[6]++;
+                }
+            }
+        }
+        for (r = 0; r < p; r++)
+            for (j = 0; j < p; j++)
+                if (wire[r * p + j] >= 0) times_sent[(j * n + wire[r * p + j]) * p + r]++;
+    }
+    for (j = 0; j < p; j++)
+        for (b = 0; b < n; b++) {
+            result[j * n + b] = value[(j * n + b) * p + j];
+            for (r = 0; r < p; r++)
+                if (r != j && times_sent[(j * n + b) * p + r] != 1) stats[4]++;
+        }
+    free(recvs); free(sends); free(wire); free(wire_val); free(times_sent);
+    return q;
+}

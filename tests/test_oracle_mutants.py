@@ -51,6 +51,19 @@ MUTANTS = [
      "value[want * p + a] = wire_val[t];"),
     ("simulated reduction: rounds not reversed", "for (i = n + q - 1 + x - 1; i >= x; i--) {",
      "for (i = x; i < n + q - 1 + x; i++) {"),
+    ("all-broadcast: the sender leaves out its own root instead of the to-processor's",
+     "if (j != t) blk = round_block_(sends[", "if (j != r) blk = round_block_(sends["),
+    ("all-broadcast: unpacked from the to-processor's message",
+     "int64_t f = (r - skip[k] + p) % p;\n            for (j = 0; j < p; j++) {\n                int64_t want;",
+     "int64_t f = (r + skip[k]) % p;\n            for (j = 0; j < p; j++) {\n                int64_t want;"),
+    ("all-broadcast: processor r reads root j's row at (j - r) mod p", "int64_t v = (r - j + p) % p;",
+     "int64_t v = (j - r + p) % p;"),
+    ("all-broadcast: blocks not shifted by the virtual rounds", "blk = (int64_t)entry + (i / q) * q - x;",
+     "blk = (int64_t)entry + (i / q) * q;"),
+    ("all-reduction: a partial result expected from a root for its own blocks", "if (j != t) want = round_block_(sends[",
+     "if (1) want = round_block_(sends["),
+    ("all-reduction: received value replaces the partial result",
+     "value[(j * n + want) * p + r] += wire_val[t * p + j];", "value[(j * n + want) * p + r] = wire_val[t * p + j];"),
 ]
 
 

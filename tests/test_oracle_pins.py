@@ -625,3 +625,93 @@ def test_simulated_reduction_notices_damaged_tables():
     assert sum(int(v) for v in stats[:5]) > 0 and (result != want).any()
     result, stats = oracle.simulate_reduce(p, (root + 1) % p, n, recv, send, value)
     assert sum(int(v) for v in stats[:5]) > 0
+
+
+# ---------------------------------------------------------------- Algorithm 7 by all processors; its reversal
+def test_simulated_allbroadcast_of_correct_tables():
+    """Observation 1 item 2 / Algorithm 7: all p broadcasts share the rounds.  Every processor ends with all
+    n blocks of every root after exactly n-1+q rounds, nothing is packed before it is held, packed and
+    unpacked blocks agree root by root, and the broadcast from root j runs exactly as Algorithm 1 alone
+    would run it (whose arrival rounds Theorem 1 pins)."""
+    for p in list(range(1, 20)) + [33, 64, 65]:
+        q = oracle.q_of(p)
+        for n in sorted({1, 2, 3, max(q, 1), q + 2}):
+            arrival, stats = oracle.simulate_allbroadcast(p, n)
+            assert list(stats[:6]) == [0] * 6, (p, n, stats)
+            assert stats[6] == (p - 1) * n * p
+            if p > 1:
+                assert stats[7] == n - 1 + q
+            for j in range(p) if p <= 19 else (0, 1, p // 2, p - 1):
+                recv, send = oracle.schedule_table(p, j)
+                alone, _ = oracle.simulate_broadcast(p, j, n, recv, send)
+                assert np.array_equal(arrival[j], alone), (p, n, j)
+            # the same from the root-0 tables read at row (r - j) mod p
+            recv0, send0 = oracle.schedule_table(p, 0)
+            arrival0, stats0 = oracle.simulate_allbroadcast(p, n, recv0, send0)
+            assert np.array_equal(arrival, arrival0) and list(stats) == list(stats0)
+
+
+def test_simulated_allbroadcast_power_of_two_single_block():
+    # p = 2^q, n = 1: processor r gets root j's block in round floor(log2((r - j) mod p)) + 1
+    for q in range(1, 7):
+        p = 2 ** q
+        arrival, stats = oracle.simulate_allbroadcast(p, 1)
+        for j in range(p):
+            for r in range(p):
+                v = (r - j) % p
+                assert arrival[j, 0, r] == (0 if v == 0 else v.bit_length()), (p, j, r)
+
+
+def test_simulated_allbroadcast_notices_damaged_tables():
+    p, n = 21, 6
+    q = oracle.q_of(p)
+    recv0, send0 = oracle.schedule_table(p, 0)
+    r2 = recv0.copy(); r2[7, 2] = q + 3                       # out of range: every (processor, root) pair with
+    _, stats = oracle.simulate_allbroadcast(p, n, r2, send0)  # (r - j) mod p = 7 reads it
+    assert stats[5] == p and stats[4] > 0
+    s2 = send0.copy(); s2[5, 1] = s2[5, 1] - 1 if s2[5, 1] > -q else s2[5, 1] + 1
+    _, stats = oracle.simulate_allbroadcast(p, n, recv0, s2)
+    assert sum(int(v) for v in stats[:5]) > 0
+    # tables of another p's shape would not even have the right size; tables of another root do
+    recv1, send1 = oracle.schedule_table(p, 1)
+    _, stats = oracle.simulate_allbroadcast(p, n, recv1, send1)
+    assert sum(int(v) for v in stats[:5]) > 0
+
+
+def test_simulated_allreduction_gives_every_root_its_sums():
+    """Observation 1 item 4: the rounds reversed.  Root j ends with the sum over all processors of the
+    contributions to each of its blocks (the definition of the reduction), every partial result of every
+    non-root processor is passed on exactly once, and root j's reduction is what the reversal of
+    Algorithm 1 alone gives."""
+    for p in list(range(1, 20)) + [33, 64, 65]:
+        q = oracle.q_of(p)
+        for n in sorted({1, 2, max(q, 1), q + 2}):
+            value = np.random.default_rng(p * 977 + n).integers(0, 2 ** 63, size=(p, n, p), dtype=np.uint64)
+            result, stats = oracle.simulate_allreduce(p, n, value)
+            with np.errstate(over="ignore"):
+                want = value.sum(axis=2, dtype=np.uint64)
+            assert np.array_equal(result, want), (p, n)
+            assert list(stats[:6]) == [0] * 6, (p, n, stats)
+            assert stats[6] == (p - 1) * n * p
+            for j in (0, p // 2, p - 1):
+                recv, send = oracle.schedule_table(p, j)
+                alone, _ = oracle.simulate_reduce(p, j, n, recv, send, value[j])
+                assert np.array_equal(result[j], alone), (p, n, j)
+            recv0, send0 = oracle.schedule_table(p, 0)
+            result0, stats0 = oracle.simulate_allreduce(p, n, value, recv0, send0)
+            assert np.array_equal(result, result0) and list(stats) == list(stats0)
+
+
+def test_simulated_allreduction_notices_damaged_tables():
+    p, n = 21, 6
+    q = oracle.q_of(p)
+    recv0, send0 = oracle.schedule_table(p, 0)
+    value = np.random.default_rng(3).integers(0, 2 ** 63, size=(p, n, p), dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        want = value.sum(axis=2, dtype=np.uint64)
+    r2 = recv0.copy(); r2[9, 1] = r2[9, 1] - 1 if r2[9, 1] > -q else r2[9, 1] + 1
+    result, stats = oracle.simulate_allreduce(p, n, value, r2, send0)
+    assert sum(int(v) for v in stats[:5]) > 0 and (result != want).any()
+    s2 = send0.copy(); s2[3, 0] = q + 1
+    _, stats = oracle.simulate_allreduce(p, n, value, recv0, s2)
+    assert stats[5] == p
