@@ -316,6 +316,64 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
                           void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
 
 /*
+ * Algorithm 7 carried out by all p processors at once (Observation 1, item 2):
+ * every processor is the root of a broadcast of its own n blocks and all p
+ * broadcasts share the n-1+q rounds.  In round i = x + j (k = i mod q) processor
+ * a packs, for every root but its to-processor (a + skip[k]) mod p, block
+ * sendblocks[root][k] + q*floor(i/q) - x, and unpacks, for every root but
+ * itself, block recvblocks[root][k] + q*floor(i/q) - x from what its
+ * from-processor (a - skip[k]) mod p packed for that root; negative blocks are
+ * neither packed nor unpacked, a block above n-1 stands for block n-1.
+ *
+ * recvblock_dev, sendblock_dev: device int32 tables [p][q] of the broadcast from
+ * root 0 as bcast_schedule(p, 0, 0, p, ...) writes them.  One pair serves every
+ * processor: its rows for root j (what bcast_allbroadcast_schedule would write
+ * for it) are the rows of rank (a - j) mod p of these tables.
+ * arrival_dev: device int32 [p][n][p], written by the call:
+ * arrival[(root*n + b)*p + a] is the round, counted from 1, in which processor a
+ * received block b of that root; 0 for a = root; -1 if it never arrived.
+ * stats_dev, delivery rule: as for bcast_simulate_broadcast, the statistics
+ * summed over all roots (correct tables: [6] = p*(p-1)*n, [7] = n-1+q).
+ * scratch_dev: at least bcast_simulate_all_scratch_bytes(p, n, 0) bytes, 16-byte
+ * aligned.  The state has p*p*n cells: sizes are the caller's to keep within
+ * its memory (p = 4096, n = 8: 512 MiB of arrival cells).
+ * Launches n-1+q small kernels per 65535 roots on cuda_stream.  Returns q.
+ */
+int64_t bcast_simulate_all_scratch_bytes(int32_t p, int64_t n, int reduction);
+int bcast_simulate_allbroadcast(int32_t p, int64_t n,
+                                const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                                int32_t *arrival_dev, uint64_t *stats_dev,
+                                void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
+
+/*
+ * The all-reduction of Observation 1, item 4 (the reduce-scatter use of the
+ * schedules): Algorithm 7's rounds from the last to the first with every
+ * communication reversed, p reductions sharing the rounds, each processor the
+ * root of the reduction of its own n blocks.  In the round that is all-broadcast
+ * round i, processor a sends to its from-processor, for every root but itself,
+ * its partial result of block recvblocks[root][k] + q*floor(i/q) - x, and
+ * receives from its to-processor t, for every root but t, a partial result of
+ * block sendblocks[root][k] + q*floor(i/q) - x, which it adds to its own.  The
+ * operator is the wrapping sum of uint64.
+ *
+ * Tables as for bcast_simulate_allbroadcast.
+ * value_dev: device uint64 [p][n][p]: value[(root*n + b)*p + a] is processor a's
+ * contribution to block b of that root on entry, partial results on return.
+ * result_dev: device uint64 [p][n]: result[root*n + b] is that root's value of
+ * its block b after the last round (correct tables: the sum over all
+ * processors; every processor ends with the n sums that are its own).
+ * stats_dev, combining rule: as for bcast_simulate_reduce, summed over all roots
+ * (correct tables: [6] = p*(p-1)*n, zeros in [0..5]).
+ * scratch_dev: at least bcast_simulate_all_scratch_bytes(p, n, 1) bytes (it
+ * holds a byte per state cell besides the byte tables), 16-byte aligned.
+ * Asynchrony, limits and return value as for bcast_simulate_allbroadcast.
+ */
+int bcast_simulate_allreduce(int32_t p, int64_t n,
+                             const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                             uint64_t *value_dev, uint64_t *result_dev, uint64_t *stats_dev,
+                             void *scratch_dev, int64_t scratch_bytes, void *cuda_stream);
+
+/*
  * Measurement aid (no counterpart in the paper): fills buffer_dev (device,
  * 16-byte aligned; bytes rounded down to a multiple of 16) with the store
  * pattern of the table kernel and nothing else -- one block of 256 threads per

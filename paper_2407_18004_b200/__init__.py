@@ -55,6 +55,10 @@ def _load():
         lib.bcast_simulate_broadcast.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_simulate_reduce.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_store_ceiling.argtypes = [vp, i64, i64, vp]
+        lib.bcast_simulate_all_scratch_bytes.argtypes = [i32, i64, ctypes.c_int]
+        lib.bcast_simulate_all_scratch_bytes.restype = i64
+        lib.bcast_simulate_allbroadcast.argtypes = [i32, i64, vp, vp, vp, vp, vp, i64, vp]
+        lib.bcast_simulate_allreduce.argtypes = [i32, i64, vp, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_round.argtypes = [i32, i64, i64, ctypes.POINTER(i32), ctypes.POINTER(i64)]
         lib.bcast_round_block.argtypes = [i32, i64, i64, vp]
         lib.bcast_round_block.restype = i64
@@ -160,6 +164,24 @@ def bcast_simulate_reduce(p: int, root: int, n: int, recvblock, sendblock, value
     nbytes = 0 if scratch is None else scratch.numel() * scratch.element_size()
     return _check(_load().bcast_simulate_reduce(p, root, n, _ptr(recvblock), _ptr(sendblock), _ptr(value),
                                                 _ptr(result), _ptr(stats), _ptr(scratch), nbytes, _stream(stream)))
+
+
+def bcast_simulate_all_scratch_bytes(p: int, n: int, reduction: bool = False) -> int:
+    return _check(_load().bcast_simulate_all_scratch_bytes(p, n, 1 if reduction else 0))
+
+
+def bcast_simulate_allbroadcast(p: int, n: int, recvblock, sendblock, arrival, stats, scratch, stream=None) -> int:
+    nbytes = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    return _check(_load().bcast_simulate_allbroadcast(p, n, _ptr(recvblock), _ptr(sendblock), _ptr(arrival),
+                                                      _ptr(stats), _ptr(scratch), nbytes, _stream(stream)))
+
+
+def bcast_simulate_allreduce(p: int, n: int, recvblock, sendblock, value, result, stats, scratch,
+                             stream=None) -> int:
+    nbytes = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    return _check(_load().bcast_simulate_allreduce(p, n, _ptr(recvblock), _ptr(sendblock), _ptr(value),
+                                                   _ptr(result), _ptr(stats), _ptr(scratch), nbytes,
+                                                   _stream(stream)))
 
 
 def bcast_allbroadcast_schedule(p: int, rank: int, root_begin: int, root_end: int, recvblocks, sendblocks,
@@ -272,4 +294,25 @@ def simulate_reduce(p: int, root: int, n: int, recvblock, sendblock, value):
     stats = torch.empty(8, dtype=torch.int64, device=value.device)
     scratch = torch.empty(bcast_simulate_scratch_bytes(p, n, True), dtype=torch.uint8, device=value.device)
     bcast_simulate_reduce(p, root, n, recvblock, sendblock, work, result, stats, scratch)
+    return result, stats
+
+
+def simulate_allbroadcast(p: int, n: int, recvblock, sendblock):
+    """Allocate state and scratch and run Algorithm 7 by all processors on root-0 tables: (arrival [p][n][p], stats)."""
+    import torch
+    arrival = torch.empty((p, n, p), dtype=torch.int32, device="cuda")
+    stats = torch.zeros(8, dtype=torch.int64, device="cuda")
+    scratch = torch.empty(max(bcast_simulate_all_scratch_bytes(p, n), 16), dtype=torch.uint8, device="cuda")
+    bcast_simulate_allbroadcast(p, n, recvblock, sendblock, arrival, stats, scratch)
+    return arrival, stats
+
+
+def simulate_allreduce(p: int, n: int, recvblock, sendblock, value):
+    """The all-reduction on root-0 tables; value [p][n][p] uint64 (as int64 tensor) is copied.  Returns (result [p][n], stats)."""
+    import torch
+    work = value.clone()
+    result = torch.empty((p, n), dtype=torch.int64, device="cuda")
+    stats = torch.zeros(8, dtype=torch.int64, device="cuda")
+    scratch = torch.empty(max(bcast_simulate_all_scratch_bytes(p, n, True), 16), dtype=torch.uint8, device="cuda")
+    bcast_simulate_allreduce(p, n, recvblock, sendblock, work, result, stats, scratch)
     return result, stats

@@ -1,6 +1,8 @@
 // Device-side use of schedule tables: Algorithm 1 of arXiv 2407.18004 run by all p
 // processors at once, round by round, on tables in device memory (bcast_simulate_broadcast),
-// and the same rounds reversed as a reduction (Observation 1, item 3: bcast_simulate_reduce).
+// the same rounds reversed as a reduction (Observation 1, item 3: bcast_simulate_reduce), and both
+// for all p roots at once (Algorithm 7 and Observation 1, items 2 and 4:
+// bcast_simulate_allbroadcast, bcast_simulate_allreduce).
 // See include/bcast_sched.h for the contracts.
 //
 // Layout and launch shape
@@ -38,6 +40,16 @@ static int host_q(int64_t p)
     int q = 0;
     while (((int64_t)1 << q) < p) ++q;
     return q;
+}
+
+// SMs of the current device (148 if the query fails: only a grid size depends on it).
+static int device_sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return 148;
+    return sms;
 }
 
 // Counters of one block: summed per warp with redux, per block in shared memory, and added
@@ -239,6 +251,132 @@ __global__ void copy_row_kernel(const uint64_t *__restrict__ value, uint64_t *__
     if (b < n) result[b] = value[b];
 }
 
+// ------------------------------------------------------------------ all roots at once (Algorithm 7 and its reversal)
+// The p broadcasts of Algorithm 7 share the rounds, and processor a's rows for root j are the
+// rows of virtual rank v = (a - j) mod p of the broadcast tables of root 0.  Thread (a, j) does
+// for root j what the kernels above do for their one root, with the byte tables read at v:
+// "packed for every root but the to-processor" is "nothing is sent to the root", "unpacked for
+// every root but oneself" is "the root receives nothing".  State: one slab of n*p cells per root.
+__global__ void __launch_bounds__(kThreads)
+init_arrival_all_kernel(int32_t *__restrict__ arrival, uint32_t p, uint32_t root0, int64_t n)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t j = root0 + blockIdx.y;
+    if (a >= p) return;
+    int32_t *slab = arrival + (size_t)j * (size_t)n * p;
+    for (int64_t b = 0; b < n; ++b) slab[(size_t)b * p + a] = a == j ? 0 : -1;
+}
+
+// Every (processor, root) pair reads one row of the given tables, and each row serves p pairs: the count
+// of entries out of range, taken once over the tables, is that of all pairs after this.
+__global__ void scale_bad_entries_kernel(unsigned long long *stats, unsigned long long p) { stats[5] *= p; }
+
+__global__ void __launch_bounds__(kThreads)
+allbroadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
+                          int32_t *arrival, uint32_t p, uint32_t root0, int64_t n, uint32_t skip_k,
+                          int64_t shift, int32_t round, unsigned long long *stats)
+{
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t j = root0 + blockIdx.y;
+    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
+    if (a < p && a != j) {
+        const uint32_t v = a >= j ? a - j : a + (p - j);                       // a's virtual rank for root j, > 0
+        const uint32_t vf = v >= skip_k ? v - skip_k : v + (p - skip_k);       // and its from-processor's
+        const uint32_t f = a >= skip_k ? a - skip_k : a + (p - skip_k);
+        int32_t *slab = arrival + (size_t)j * (size_t)n * p;
+        const int64_t want = block_of(recv_k[v], shift, n);
+        const int64_t sent = block_of(send_k[vf], shift, n);                   // f's to-processor is a, not the root
+        if (want < 0) {
+            if (sent >= 0) c3 = 1;
+        } else if (sent != want) {
+            c0 = 1;
+        } else {
+            const int32_t at_f = slab[(size_t)want * p + f];
+            const int32_t at_a = slab[(size_t)want * p + a];
+            if (!(at_f >= 0 && at_f < round)) c1 = 1;
+            else if (at_a >= 0) c2 = 1;
+            else { slab[(size_t)want * p + a] = round; c6 = 1; }
+        }
+    }
+    add_stat(bstats, 0, c0);
+    add_stat(bstats, 1, c1);
+    add_stat(bstats, 2, c2);
+    add_stat(bstats, 3, c3);
+    add_stat(bstats, 6, c6);
+    if (__any_sync(0xffffffffu, c6 != 0u) && (threadIdx.x & 31) == 0) bstats.last_round = (unsigned int)round;
+    stats_end(bstats, stats);
+}
+
+// One all-reduction round: thread (a, j) as reduce_round_kernel's thread a with root j.
+__global__ void __launch_bounds__(kThreads)
+allreduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
+                       uint64_t *value, uint8_t *sent, uint32_t p, uint32_t root0, int64_t n,
+                       uint32_t skip_k, int64_t shift, unsigned long long *stats)
+{
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t j = root0 + blockIdx.y;
+    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
+    if (a < p) {
+        uint32_t t = a + skip_k;
+        if (t >= p) t -= p;
+        const uint32_t v = a >= j ? a - j : a + (p - j);
+        uint32_t vt = v + skip_k;
+        if (vt >= p) vt -= p;
+        uint64_t *val = value + (size_t)j * (size_t)n * p;
+        uint8_t *snt = sent + (size_t)j * (size_t)n * p;
+        const int64_t mine = a == j ? -1 : block_of(recv_k[v], shift, n);          // what a sends
+        const int64_t got = t == j ? -1 : block_of(recv_k[vt], shift, n);          // what t sends to a
+        const int64_t want = t == j ? -1 : block_of(send_k[v], shift, n);
+        uint8_t sent_mine = 0;
+        if (mine >= 0) {
+            sent_mine = snt[(size_t)mine * p + a];
+            if (sent_mine > 0) c2 = 1;
+        }
+        if (want < 0) {
+            if (got >= 0) c3 = 1;
+        } else if (got != want) {
+            c0 = 1;
+        } else if (a != j && (mine == want || snt[(size_t)want * p + a] > 0)) {
+            c1 = 1;
+        } else {
+            val[(size_t)want * p + a] += val[(size_t)want * p + t];
+            c6 = 1;
+        }
+        if (mine >= 0 && sent_mine < 2) snt[(size_t)mine * p + a] = sent_mine + 1;
+    }
+    add_stat(bstats, 0, c0);
+    add_stat(bstats, 1, c1);
+    add_stat(bstats, 2, c2);
+    add_stat(bstats, 3, c3);
+    add_stat(bstats, 6, c6);
+    stats_end(bstats, stats);
+}
+
+__global__ void __launch_bounds__(kThreads)
+allreduce_finish_kernel(const uint64_t *__restrict__ value, const uint8_t *__restrict__ sent,
+                        uint64_t *__restrict__ result, uint32_t p, uint32_t root0, int64_t n,
+                        unsigned long long *stats)
+{
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const uint32_t j = root0 + blockIdx.y;
+    unsigned int c4 = 0;
+    if (a < p) {
+        const size_t slab = (size_t)j * (size_t)n * p;
+        for (int64_t b = 0; b < n; ++b) {
+            if (a == j) result[(size_t)j * n + b] = value[slab + (size_t)b * p + a];
+            else if (sent[slab + (size_t)b * p + a] != 1) c4 += 1;
+        }
+    }
+    add_stat(bstats, 4, c4);
+    stats_end(bstats, stats);
+}
+
 struct Plan {
     int q;
     int64_t P;
@@ -332,7 +470,8 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
     }
     const size_t cells = (size_t)n * (size_t)p;
     const size_t want_blocks = (cells + kThreads - 1) / kThreads;
-    count_missing_kernel<<<(unsigned int)(want_blocks < 148 * 16 ? want_blocks : 148 * 16), kThreads, 0, stream>>>(
+    const size_t most = (size_t)device_sm_count() * 16;
+    count_missing_kernel<<<(unsigned int)(want_blocks < most ? want_blocks : most), kThreads, 0, stream>>>(
         arrival_dev, cells, stats);
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
@@ -379,6 +518,118 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
         const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
         reduce_finish_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(
             value_dev + (size_t)b0 * p, sent + (size_t)b0 * p, result_dev + b0, (uint32_t)p, (uint32_t)root, stats);
+    }
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return q;
+}
+
+int64_t bcast_simulate_all_scratch_bytes(int32_t p, int64_t n, int reduction)
+{
+    if (p < 1) return BCAST_EINVAL_P;
+    if (n < 1) return BCAST_EINVAL_N;
+    const int q = host_q(p);
+    int64_t bytes = kHeaderBytes + 2 * (int64_t)q * padded(p);
+    if (reduction) bytes += (int64_t)p * n * (int64_t)p;           // sent counts, a byte per (root, block, processor)
+    return bytes;
+}
+
+int bcast_simulate_allbroadcast(int32_t p, int64_t n,
+                                const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                                int32_t *arrival_dev, uint64_t *stats_dev,
+                                void *scratch_dev, int64_t scratch_bytes, void *cuda_stream)
+{
+    const int rc = check_common(p, 0, n, recvblock_dev, sendblock_dev, arrival_dev, stats_dev);
+    if (rc != BCAST_OK) return rc;
+    if ((uintptr_t)arrival_dev & 3u) return BCAST_EALIGN;
+    const Plan plan = make_plan(p, n);
+    const int q = plan.q;
+    if (q > 0) {
+        if (scratch_dev == nullptr) return BCAST_ENULL;
+        if ((uintptr_t)scratch_dev & 15u) return BCAST_EALIGN;
+        if (scratch_bytes < bcast_simulate_all_scratch_bytes(p, n, 0)) return BCAST_ESCRATCH;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long *stats = reinterpret_cast<unsigned long long *>(stats_dev);
+    if (cudaMemsetAsync(stats_dev, 0, 8 * sizeof(uint64_t), stream) != cudaSuccess) return BCAST_ECUDA;
+    const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
+    // the roots go in slices of at most 65535 (the grid's y limit)
+    for (int64_t j0 = 0; j0 < p; j0 += 65535) {
+        const unsigned int nj = (unsigned int)(p - j0 < 65535 ? p - j0 : 65535);
+        init_arrival_all_kernel<<<dim3(blocks, nj), kThreads, 0, stream>>>(arrival_dev, (uint32_t)p, (uint32_t)j0, n);
+    }
+    if (q > 0) {
+        int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
+        int8_t *send_t = recv_t + (size_t)q * plan.P;
+        transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
+            recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
+        scale_bad_entries_kernel<<<1, 1, 0, stream>>>(stats, (unsigned long long)p);
+        const int64_t rounds = n - 1 + q;
+        for (int64_t jr = 0; jr < rounds; ++jr) {
+            const int64_t i = plan.x + jr;
+            const int k = (int)(i % q);
+            const int64_t shift = (i / q) * q - plan.x;
+            for (int64_t j0 = 0; j0 < p; j0 += 65535) {
+                const unsigned int nj = (unsigned int)(p - j0 < 65535 ? p - j0 : 65535);
+                allbroadcast_round_kernel<<<dim3(blocks, nj), kThreads, 0, stream>>>(
+                    recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, (uint32_t)p,
+                    (uint32_t)j0, n, plan.skip[k], shift, (int32_t)(jr + 1), stats);
+            }
+        }
+    }
+    const size_t cells = (size_t)p * (size_t)n * (size_t)p;
+    const size_t want_blocks = (cells + kThreads - 1) / kThreads;
+    const size_t most = (size_t)device_sm_count() * 16;
+    count_missing_kernel<<<(unsigned int)(want_blocks < most ? want_blocks : most), kThreads, 0, stream>>>(
+        arrival_dev, cells, stats);
+    if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
+    return q;
+}
+
+int bcast_simulate_allreduce(int32_t p, int64_t n,
+                             const int32_t *recvblock_dev, const int32_t *sendblock_dev,
+                             uint64_t *value_dev, uint64_t *result_dev, uint64_t *stats_dev,
+                             void *scratch_dev, int64_t scratch_bytes, void *cuda_stream)
+{
+    const int rc = check_common(p, 0, n, recvblock_dev, sendblock_dev, value_dev, stats_dev);
+    if (rc != BCAST_OK) return rc;
+    if (result_dev == nullptr) return BCAST_ENULL;
+    if (((uintptr_t)value_dev & 7u) || ((uintptr_t)result_dev & 7u)) return BCAST_EALIGN;
+    const Plan plan = make_plan(p, n);
+    const int q = plan.q;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    unsigned long long *stats = reinterpret_cast<unsigned long long *>(stats_dev);
+    if (cudaMemsetAsync(stats_dev, 0, 8 * sizeof(uint64_t), stream) != cudaSuccess) return BCAST_ECUDA;
+    if (q == 0) {
+        copy_row_kernel<<<(unsigned int)((n + 255) / 256), 256, 0, stream>>>(value_dev, result_dev, n);
+        return cudaGetLastError() == cudaSuccess ? 0 : BCAST_ECUDA;
+    }
+    if (scratch_dev == nullptr) return BCAST_ENULL;
+    if ((uintptr_t)scratch_dev & 15u) return BCAST_EALIGN;
+    if (scratch_bytes < bcast_simulate_all_scratch_bytes(p, n, 1)) return BCAST_ESCRATCH;
+    int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
+    int8_t *send_t = recv_t + (size_t)q * plan.P;
+    uint8_t *sent = reinterpret_cast<uint8_t *>(send_t + (size_t)q * plan.P);
+    if (cudaMemsetAsync(sent, 0, (size_t)p * (size_t)n * (size_t)p, stream) != cudaSuccess) return BCAST_ECUDA;
+    const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
+    transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
+        recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
+    scale_bad_entries_kernel<<<1, 1, 0, stream>>>(stats, (unsigned long long)p);
+    const int64_t rounds = n - 1 + q;
+    for (int64_t jr = rounds - 1; jr >= 0; --jr) {                 // the all-broadcast's rounds, last one first
+        const int64_t i = plan.x + jr;
+        const int k = (int)(i % q);
+        const int64_t shift = (i / q) * q - plan.x;
+        for (int64_t j0 = 0; j0 < p; j0 += 65535) {
+            const unsigned int nj = (unsigned int)(p - j0 < 65535 ? p - j0 : 65535);
+            allreduce_round_kernel<<<dim3(blocks, nj), kThreads, 0, stream>>>(
+                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, value_dev, sent, (uint32_t)p, (uint32_t)j0,
+                n, plan.skip[k], shift, stats);
+        }
+    }
+    for (int64_t j0 = 0; j0 < p; j0 += 65535) {
+        const unsigned int nj = (unsigned int)(p - j0 < 65535 ? p - j0 : 65535);
+        allreduce_finish_kernel<<<dim3(blocks, nj), kThreads, 0, stream>>>(value_dev, sent, result_dev, (uint32_t)p,
+                                                                           (uint32_t)j0, n, stats);
     }
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;

@@ -1,5 +1,6 @@
 """GPU parity of the entry points that USE schedule tables: Algorithm 1 run by all processors
-(bcast_simulate_broadcast), its reversal as a reduction (bcast_simulate_reduce), and the tables
+(bcast_simulate_broadcast), its reversal as a reduction (bcast_simulate_reduce), both for all p roots at
+once (Algorithm 7: bcast_simulate_allbroadcast, bcast_simulate_allreduce), and the tables
 with Algorithm 1's preamble applied (bcast_schedule_shifted).  All through the C ABI, bit for bit
 against the CPU oracle on the same tables."""
 import numpy as np
@@ -235,3 +236,83 @@ def test_more_blocks_than_one_launch_grid_holds():
     with np.errstate(over="ignore"):
         assert result.tolist() == value.sum(axis=1, dtype=np.uint64).tolist()
     assert rstats[:6].tolist() == [0] * 6
+
+
+# ------------------------------------------------------------------ all roots at once: Algorithm 7 and its reversal
+def check_all(p, n, recv0, send0, tables_from_algorithm7):
+    """The device gets the root-0 tables; the oracle takes every processor's tables from Algorithm 7's own
+    loops (correct tables) or reads the same given tables at row (r - j) mod p (damaged tables)."""
+    given = (None, None) if tables_from_algorithm7 else (recv0, send0)
+    want_arrival, want_stats = oracle.simulate_allbroadcast(p, n, *given)
+    d_recv, d_send = (dev(recv0), dev(send0)) if p > 1 else (None, None)
+    arrival, stats = bs.simulate_allbroadcast(p, n, d_recv, d_send)
+    value = np.random.default_rng(p * 31 + n).integers(0, 2 ** 63, size=(p, n, p), dtype=np.uint64)
+    want_result, want_rstats = oracle.simulate_allreduce(p, n, value, *given)
+    result, rstats = bs.simulate_allreduce(p, n, d_recv, d_send, dev(value.view(np.int64)))
+    torch.cuda.synchronize()
+    assert u64(stats).tolist() == want_stats.tolist()
+    assert np.array_equal(arrival.cpu().numpy(), want_arrival)
+    assert u64(rstats).tolist() == want_rstats.tolist()
+    assert np.array_equal(u64(result), want_result)
+    return want_stats, want_rstats, value, want_result
+
+
+@pytest.mark.parametrize("p", [1, 2, 3, 9, 17, 18, 64, 100, 257])
+def test_allbroadcast_and_allreduction_every_phase_offset(p):
+    q = oracle.q_of(p)
+    recv0, send0 = oracle.schedule_table(p, 0)
+    for n in sorted({1, 2, max(q, 1), q + 1, 2 * q + 3}):
+        stats, rstats, value, result = check_all(p, n, recv0, send0, True)
+        assert stats[:6].tolist() == [0] * 6 and stats[6] == p * (p - 1) * n
+        assert rstats[:6].tolist() == [0] * 6 and rstats[6] == p * (p - 1) * n
+        with np.errstate(over="ignore"):
+            assert np.array_equal(result, value.sum(axis=2, dtype=np.uint64))
+
+
+def test_allbroadcast_and_allreduction_on_device_tables():
+    # the tables the library itself wrote, p large enough for several blocks of processors and of roots
+    p, n = 1500, 5
+    q = bs.bcast_q(p)
+    recv, send = bs.schedule(p, 0)
+    arrival, stats = bs.simulate_allbroadcast(p, n, recv, send)
+    value = torch.randint(0, 2 ** 62, (p, n, p), dtype=torch.int64, device="cuda",
+                          generator=torch.Generator(device="cuda").manual_seed(1))
+    result, rstats = bs.simulate_allreduce(p, n, recv, send, value)
+    torch.cuda.synchronize()
+    assert u64(stats).tolist() == [0, 0, 0, 0, 0, 0, p * (p - 1) * n, n - 1 + q]
+    assert u64(rstats).tolist() == [0, 0, 0, 0, 0, 0, p * (p - 1) * n, 0]
+    assert bool((result == value.sum(dim=2)).all())
+    # root j's slab is Algorithm 1 alone from root j
+    for j in (0, 700, p - 1):
+        orecv, osend = oracle.schedule_table(p, j)
+        alone, _ = oracle.simulate_broadcast(p, j, n, orecv, osend)
+        assert np.array_equal(arrival[j].cpu().numpy(), alone)
+
+
+def test_allbroadcast_and_allreduction_on_damaged_tables():
+    p, n = 45, 7
+    q = oracle.q_of(p)
+    recv0, send0 = oracle.schedule_table(p, 0)
+    r2 = recv0.copy(); r2[7, 2] = q + 3
+    stats, rstats, _, _ = check_all(p, n, r2, send0, False)
+    assert stats[5] == p and rstats[5] == p
+    s2 = send0.copy(); s2[5, 1] = s2[5, 1] - 1 if s2[5, 1] > -q else s2[5, 1] + 1
+    stats, rstats, _, _ = check_all(p, n, recv0, s2, False)
+    assert sum(int(v) for v in stats[:5]) > 0 and sum(int(v) for v in rstats[:5]) > 0
+    recv1, send1 = oracle.schedule_table(p, 1)
+    stats, _, _, _ = check_all(p, n, recv1, send1, False)
+    assert sum(int(v) for v in stats[:5]) > 0
+
+
+def test_allbroadcast_argument_errors():
+    p, n = 17, 3
+    recv, send = bs.schedule(p, 0)
+    arrival = torch.empty((p, n, p), dtype=torch.int32, device="cuda")
+    stats = torch.zeros(8, dtype=torch.int64, device="cuda")
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bs.BcastError):
+        bs.bcast_simulate_allbroadcast(p, n, recv, send, arrival, stats, small)
+    with pytest.raises(bs.BcastError):
+        bs.bcast_simulate_allbroadcast(p, 0, recv, send, arrival, stats, small)
+    with pytest.raises(bs.BcastError):
+        bs.bcast_simulate_allreduce(p, n, recv, send, None, None, stats, small)
