@@ -269,7 +269,8 @@ int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev
  * Correct tables give zeros in [0..5].
  * scratch_dev: device memory, 16-byte aligned, at least
  * bcast_simulate_scratch_bytes(p, n, 0) bytes; it receives round-major byte
- * copies of the tables.  Contents after the call are unspecified.
+ * copies of the tables and a bit per (processor, block) for who holds what.
+ * Contents after the call are unspecified.
  * Launches n-1+q small kernels on cuda_stream, asynchronously.  Returns q.
  * Limits: n < 2^31 - 64; n * p int32 cells must fit the caller's memory.
  */

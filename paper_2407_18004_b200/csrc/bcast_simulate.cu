@@ -34,6 +34,7 @@ constexpr int8_t kInvalid = -128;
 constexpr int64_t kHeaderBytes = 256;
 
 __host__ __device__ inline int64_t padded(int64_t p) { return (p + 127) / 128 * 128; }
+inline int64_t set_words(int64_t n) { return (n + 63) / 64; }      // 64-bit words of a bit set over n blocks
 
 static int host_q(int64_t p)
 {
@@ -118,6 +119,23 @@ init_arrival_kernel(int32_t *__restrict__ arrival, uint32_t p, uint32_t root)
     if (a < p) arrival[(size_t)blockIdx.y * p + a] = a == root ? 0 : -1;
 }
 
+// Bit sets over the blocks, a word of 64 blocks per processor: set[w * P + a].  Cleared for everybody
+// and, where `root_full`, filled with the n blocks for the root.
+__global__ void __launch_bounds__(kThreads)
+init_block_sets_kernel(unsigned long long *__restrict__ set, size_t P, uint32_t p, uint32_t root, int64_t n,
+                       int root_full)
+{
+    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
+    const int64_t w = blockIdx.y;
+    if (a >= P) return;
+    unsigned long long word = 0ull;
+    if (root_full && a == root && a < p) {
+        const int64_t left = n - 64 * w;
+        word = left >= 64 ? ~0ull : ((1ull << left) - 1ull);
+    }
+    set[(size_t)w * P + a] = word;
+}
+
 // Block of a table entry in a round: entry + shift, nothing (-1) when negative or invalid,
 // n-1 when above it.
 __device__ __forceinline__ int64_t block_of(int8_t entry, int64_t shift, int64_t n)
@@ -130,30 +148,50 @@ __device__ __forceinline__ int64_t block_of(int8_t entry, int64_t shift, int64_t
 
 // One communication round of Algorithm 1 for every processor: skip index k (the rows of the
 // byte tables passed in), blocks = entry + shift, `round` counted from 1.
+//
+// Who holds what is kept twice: arrival[b][a], the result, written once per delivery, and
+// held[w][a], a bit per block, which is what the round reads (8 bytes per processor, consecutive
+// processors side by side, where the arrival cells of a round lie in up to 2q different rows).
+// Thread a alone writes a's word.  A reader of f's word asks whether f held the block BEFORE the
+// round; the bit can only be about to change in this round if f is itself receiving that very
+// block now, and then the answer is taken from f's arrival cell, which is -1 or >= round for
+// anything not held before, whether or not f's write is seen.
 __global__ void __launch_bounds__(kThreads)
 broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
-                       int32_t *arrival, uint32_t p, uint32_t root, int64_t n, uint32_t skip_k,
-                       int64_t shift, int32_t round, unsigned long long *stats)
+                       int32_t *arrival, unsigned long long *held, size_t P, uint32_t p, uint32_t root,
+                       int64_t n, uint32_t skip_k, int64_t shift, int32_t round, unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
-    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
-    if (a < p && a != root) {
+    // a resident grid strides over the processors: a few thousand blocks would each add their
+    // counters to the same statistics words, and those atomics would set the pace of the round
+    for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
+        if (a == root) continue;
         const uint32_t f = a >= skip_k ? a - skip_k : a + (p - skip_k);     // from-processor
         const int64_t want = block_of(recv_k[a], shift, n);
         // f's to-processor is a, which is not the root, so f's send is not suppressed
         const int64_t sent = block_of(send_k[f], shift, n);
         if (want < 0) {
-            if (sent >= 0) c3 = 1;
+            if (sent >= 0) c3 += 1;
         } else if (sent != want) {
-            c0 = 1;
+            c0 += 1;
         } else {
-            const int32_t at_f = arrival[(size_t)want * p + f];
-            const int32_t at_a = arrival[(size_t)want * p + a];
-            if (!(at_f >= 0 && at_f < round)) c1 = 1;                        // not held before the round
-            else if (at_a >= 0) c2 = 1;
-            else { arrival[(size_t)want * p + a] = round; c6 = 1; }
+            const size_t word = (size_t)(want >> 6) * P;
+            const unsigned long long bit = 1ull << (want & 63);
+            bool f_held = (held[word + f] & bit) != 0ull;
+            if (f_held && f != root && block_of(recv_k[f], shift, n) == want) {
+                const int32_t at_f = arrival[(size_t)want * p + f];          // f may be getting it only now
+                f_held = at_f >= 0 && at_f < round;
+            }
+            const unsigned long long mine = held[word + a];
+            if (!f_held) c1 += 1;                                            // not held before the round
+            else if ((mine & bit) != 0ull) c2 += 1;
+            else {
+                held[word + a] = mine | bit;
+                arrival[(size_t)want * p + a] = round;
+                c6 += 1;
+            }
         }
     }
     add_stat(bstats, 0, c0);
@@ -177,6 +215,23 @@ count_missing_kernel(const int32_t *__restrict__ arrival, size_t cells, unsigned
     stats_end(bstats, stats);
 }
 
+// (processor, block) pairs still missing, from the bit sets (a bit is set exactly when the arrival
+// cell is): word w of a processor covers min(64, n - 64 w) blocks.
+__global__ void __launch_bounds__(kThreads)
+count_missing_sets_kernel(const unsigned long long *__restrict__ held, size_t P, uint32_t p, int64_t n,
+                          unsigned long long *stats)
+{
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
+    const int64_t w = blockIdx.y;
+    const int in_word = (int)(n - 64 * w >= 64 ? 64 : n - 64 * w);
+    unsigned int missing = 0;
+    for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads)
+        missing += (unsigned int)(in_word - __popcll(held[(size_t)w * P + a]));
+    add_stat(bstats, 4, missing);
+    stats_end(bstats, stats);
+}
+
 // ------------------------------------------------------------------ reduction (reversed rounds)
 // One reduction round for every processor.  Processor a sends its partial result of the block
 // it RECEIVED in the corresponding broadcast round to its from-processor (the root sends
@@ -190,35 +245,40 @@ count_missing_kernel(const int32_t *__restrict__ arrival, size_t cells, unsigned
 // which is counted instead); sent[.][a] is read and written by thread a alone.
 __global__ void __launch_bounds__(kThreads)
 reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
-                    uint64_t *value, uint8_t *sent, uint32_t p, uint32_t root, int64_t n,
-                    uint32_t skip_k, int64_t shift, unsigned long long *stats)
+                    uint64_t *value, unsigned long long *once, unsigned long long *twice, size_t P,
+                    uint32_t p, uint32_t root, int64_t n, uint32_t skip_k, int64_t shift,
+                    unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
-    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
-    if (a < p) {
+    for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
         uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
         if (t >= p) t -= p;
         const int64_t mine = a == root ? -1 : block_of(recv_k[a], shift, n);       // what a sends
         const int64_t got = t == root ? -1 : block_of(recv_k[t], shift, n);        // what t sends to a
         const int64_t want = t == root ? -1 : block_of(send_k[a], shift, n);
-        uint8_t sent_mine = 0;
+        // how often a has sent a block: bit in once[] after the first time, in twice[] after the second;
+        // thread a alone reads and writes a's words
+        bool sent_mine = false;
         if (mine >= 0) {
-            sent_mine = sent[(size_t)mine * p + a];
-            if (sent_mine > 0) c2 = 1;
+            sent_mine = (once[(size_t)(mine >> 6) * P + a] >> (mine & 63)) & 1ull;
+            if (sent_mine) c2 += 1;
         }
         if (want < 0) {
-            if (got >= 0) c3 = 1;
+            if (got >= 0) c3 += 1;
         } else if (got != want) {
-            c0 = 1;
-        } else if (a != root && (mine == want || sent[(size_t)want * p + a] > 0)) {
-            c1 = 1;                                        // it would never be passed on
+            c0 += 1;
+        } else if (a != root && (mine == want || ((once[(size_t)(want >> 6) * P + a] >> (want & 63)) & 1ull))) {
+            c1 += 1;                                       // it would never be passed on
         } else {
             value[(size_t)want * p + a] += value[(size_t)want * p + t];
-            c6 = 1;
+            c6 += 1;
         }
-        if (mine >= 0 && sent_mine < 2) sent[(size_t)mine * p + a] = sent_mine + 1;
+        if (mine >= 0) {
+            unsigned long long *set = sent_mine ? twice : once;
+            set[(size_t)(mine >> 6) * P + a] |= 1ull << (mine & 63);
+        }
     }
     add_stat(bstats, 0, c0);
     add_stat(bstats, 1, c1);
@@ -229,17 +289,23 @@ reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict_
 }
 
 __global__ void __launch_bounds__(kThreads)
-reduce_finish_kernel(const uint64_t *__restrict__ value, const uint8_t *__restrict__ sent,
-                     uint64_t *__restrict__ result, uint32_t p, uint32_t root, unsigned long long *stats)
+reduce_finish_kernel(const uint64_t *__restrict__ value, const unsigned long long *__restrict__ once,
+                     const unsigned long long *__restrict__ twice, size_t P, uint64_t *__restrict__ result,
+                     uint32_t p, uint32_t root, int64_t b0, unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
     const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
-    const size_t b = blockIdx.y;
+    const int64_t b = b0 + blockIdx.y;
     unsigned int c4 = 0;
     if (a < p) {
-        if (a == root) result[b] = value[b * p + a];
-        else if (sent[b * p + a] != 1) c4 = 1;
+        if (a == root) {
+            result[b] = value[(size_t)b * p + a];
+        } else {
+            const bool sent_once = (once[(size_t)(b >> 6) * P + a] >> (b & 63)) & 1ull;
+            const bool sent_twice = (twice[(size_t)(b >> 6) * P + a] >> (b & 63)) & 1ull;
+            if (!sent_once || sent_twice) c4 = 1;           // not exactly once
+        }
     }
     add_stat(bstats, 4, c4);
     stats_end(bstats, stats);
@@ -423,9 +489,9 @@ int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction)
     if (n < 1) return BCAST_EINVAL_N;
     const int q = host_q(p);
     const int64_t P = padded(p);
-    int64_t bytes = kHeaderBytes + 2 * (int64_t)q * P;
-    if (reduction) bytes += n * (int64_t)p;                        // sent counts
-    return bytes;
+    // byte tables, then bit sets over the blocks (8 bytes per processor and 64 blocks): who holds what
+    // (broadcast), or what was sent once and what twice (reduction)
+    return kHeaderBytes + 2 * (int64_t)q * P + (reduction ? 2 : 1) * set_words(n) * P * 8;
 }
 
 int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
@@ -456,23 +522,37 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
     if (q > 0) {
         int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
         int8_t *send_t = recv_t + (size_t)q * plan.P;
+        unsigned long long *held = reinterpret_cast<unsigned long long *>(send_t + (size_t)q * plan.P);
+        const unsigned int pblocks = (unsigned int)(plan.P / kThreads + (plan.P % kThreads != 0));
+        for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
+            const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
+            init_block_sets_kernel<<<dim3(pblocks, nw), kThreads, 0, stream>>>(
+                held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, (uint32_t)root, n - 64 * w0, 1);
+        }
         transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
             recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
         const int64_t rounds = n - 1 + q;
+        const unsigned int resident = (unsigned int)device_sm_count() * 8u;
+        const unsigned int round_blocks = blocks < resident ? blocks : resident;
         for (int64_t j = 0; j < rounds; ++j) {
             const int64_t i = plan.x + j;
             const int k = (int)(i % q);
             const int64_t shift = (i / q) * q - plan.x;            // Theorem 1
-            broadcast_round_kernel<<<blocks, kThreads, 0, stream>>>(
-                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, (uint32_t)p,
-                (uint32_t)root, n, plan.skip[k], shift, (int32_t)(j + 1), stats);
+            broadcast_round_kernel<<<round_blocks, kThreads, 0, stream>>>(
+                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, held, (size_t)plan.P,
+                (uint32_t)p, (uint32_t)root, n, plan.skip[k], shift, (int32_t)(j + 1), stats);
         }
     }
-    const size_t cells = (size_t)n * (size_t)p;
-    const size_t want_blocks = (cells + kThreads - 1) / kThreads;
-    const size_t most = (size_t)device_sm_count() * 16;
-    count_missing_kernel<<<(unsigned int)(want_blocks < most ? want_blocks : most), kThreads, 0, stream>>>(
-        arrival_dev, cells, stats);
+    if (q > 0) {
+        const unsigned long long *held = reinterpret_cast<const unsigned long long *>(
+            reinterpret_cast<const int8_t *>(scratch_dev) + kHeaderBytes + 2 * (size_t)q * plan.P);
+        const unsigned int resident = (unsigned int)device_sm_count() * 8u;
+        for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
+            const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
+            count_missing_sets_kernel<<<dim3(blocks < resident ? blocks : resident, nw), kThreads, 0, stream>>>(
+                held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, n - 64 * w0, stats);
+        }
+    }
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
 }
@@ -500,24 +580,27 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
     if (scratch_bytes < bcast_simulate_scratch_bytes(p, n, 1)) return BCAST_ESCRATCH;
     int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
     int8_t *send_t = recv_t + (size_t)q * plan.P;
-    uint8_t *sent = reinterpret_cast<uint8_t *>(send_t + (size_t)q * plan.P);
-    if (cudaMemsetAsync(sent, 0, (size_t)n * (size_t)p, stream) != cudaSuccess) return BCAST_ECUDA;
+    unsigned long long *once = reinterpret_cast<unsigned long long *>(send_t + (size_t)q * plan.P);
+    unsigned long long *twice = once + (size_t)set_words(n) * plan.P;
+    if (cudaMemsetAsync(once, 0, (size_t)2 * set_words(n) * plan.P * 8, stream) != cudaSuccess) return BCAST_ECUDA;
     const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
     transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
         recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
     const int64_t rounds = n - 1 + q;
+    const unsigned int resident = (unsigned int)device_sm_count() * 8u;
+    const unsigned int round_blocks = blocks < resident ? blocks : resident;
     for (int64_t j = rounds - 1; j >= 0; --j) {                    // the broadcast's rounds, last one first
         const int64_t i = plan.x + j;
         const int k = (int)(i % q);
         const int64_t shift = (i / q) * q - plan.x;
-        reduce_round_kernel<<<blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P,
-                                                             value_dev, sent, (uint32_t)p, (uint32_t)root, n,
-                                                             plan.skip[k], shift, stats);
+        reduce_round_kernel<<<round_blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P,
+                                                             value_dev, once, twice, (size_t)plan.P, (uint32_t)p,
+                                                             (uint32_t)root, n, plan.skip[k], shift, stats);
     }
     for (int64_t b0 = 0; b0 < n; b0 += 65535) {
         const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
         reduce_finish_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(
-            value_dev + (size_t)b0 * p, sent + (size_t)b0 * p, result_dev + b0, (uint32_t)p, (uint32_t)root, stats);
+            value_dev, once, twice, (size_t)plan.P, result_dev, (uint32_t)p, (uint32_t)root, b0, stats);
     }
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
