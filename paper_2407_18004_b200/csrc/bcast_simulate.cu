@@ -146,6 +146,14 @@ __device__ __forceinline__ int64_t block_of(int8_t entry, int64_t shift, int64_t
     return raw > n - 1 ? n - 1 : raw;
 }
 
+// The same in 32 bits for the kernels that run once per round over all processors (n < 2^31 - 64 and
+// shift <= n - 1, so entry + shift does not overflow); last = n - 1.
+__device__ __forceinline__ int block32(int8_t entry, int shift, int last)
+{
+    const int raw = min((int)entry + shift, last);
+    return entry == kInvalid || raw < 0 ? -1 : raw;
+}
+
 // One communication round of Algorithm 1 for every processor: skip index k (the rows of the
 // byte tables passed in), blocks = entry + shift, `round` counted from 1.
 //
@@ -159,7 +167,7 @@ __device__ __forceinline__ int64_t block_of(int8_t entry, int64_t shift, int64_t
 __global__ void __launch_bounds__(kThreads)
 broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
                        int32_t *arrival, unsigned long long *held, size_t P, uint32_t p, uint32_t root,
-                       int64_t n, uint32_t skip_k, int64_t shift, int32_t round, unsigned long long *stats)
+                       int last, uint32_t skip_k, int shift, int32_t round, unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
@@ -169,26 +177,26 @@ broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restri
     for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
         if (a == root) continue;
         const uint32_t f = a >= skip_k ? a - skip_k : a + (p - skip_k);     // from-processor
-        const int64_t want = block_of(recv_k[a], shift, n);
+        const int want = block32(recv_k[a], shift, last);
         // f's to-processor is a, which is not the root, so f's send is not suppressed
-        const int64_t sent = block_of(send_k[f], shift, n);
+        const int sent = block32(send_k[f], shift, last);
         if (want < 0) {
-            if (sent >= 0) c3 += 1;
+            c3 += sent >= 0 ? 1u : 0u;
         } else if (sent != want) {
             c0 += 1;
         } else {
-            const size_t word = (size_t)(want >> 6) * P;
+            unsigned long long *words = held + (size_t)(want >> 6) * P;
             const unsigned long long bit = 1ull << (want & 63);
-            bool f_held = (held[word + f] & bit) != 0ull;
-            if (f_held && f != root && block_of(recv_k[f], shift, n) == want) {
+            bool f_held = (words[f] & bit) != 0ull;
+            if (f_held && f != root && block32(recv_k[f], shift, last) == want) {
                 const int32_t at_f = arrival[(size_t)want * p + f];          // f may be getting it only now
                 f_held = at_f >= 0 && at_f < round;
             }
-            const unsigned long long mine = held[word + a];
+            const unsigned long long mine = words[a];
             if (!f_held) c1 += 1;                                            // not held before the round
             else if ((mine & bit) != 0ull) c2 += 1;
             else {
-                held[word + a] = mine | bit;
+                words[a] = mine | bit;
                 arrival[(size_t)want * p + a] = round;
                 c6 += 1;
             }
@@ -246,7 +254,7 @@ count_missing_sets_kernel(const unsigned long long *__restrict__ held, size_t P,
 __global__ void __launch_bounds__(kThreads)
 reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
                     uint64_t *value, unsigned long long *once, unsigned long long *twice, size_t P,
-                    uint32_t p, uint32_t root, int64_t n, uint32_t skip_k, int64_t shift,
+                    uint32_t p, uint32_t root, int last, uint32_t skip_k, int shift,
                     unsigned long long *stats)
 {
     __shared__ BlockStats bstats;
@@ -255,9 +263,9 @@ reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict_
     for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
         uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
         if (t >= p) t -= p;
-        const int64_t mine = a == root ? -1 : block_of(recv_k[a], shift, n);       // what a sends
-        const int64_t got = t == root ? -1 : block_of(recv_k[t], shift, n);        // what t sends to a
-        const int64_t want = t == root ? -1 : block_of(send_k[a], shift, n);
+        const int mine = a == root ? -1 : block32(recv_k[a], shift, last);         // what a sends
+        const int got = t == root ? -1 : block32(recv_k[t], shift, last);          // what t sends to a
+        const int want = t == root ? -1 : block32(send_k[a], shift, last);
         // how often a has sent a block: bit in once[] after the first time, in twice[] after the second;
         // thread a alone reads and writes a's words
         bool sent_mine = false;
@@ -540,7 +548,7 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
             const int64_t shift = (i / q) * q - plan.x;            // Theorem 1
             broadcast_round_kernel<<<round_blocks, kThreads, 0, stream>>>(
                 recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, held, (size_t)plan.P,
-                (uint32_t)p, (uint32_t)root, n, plan.skip[k], shift, (int32_t)(j + 1), stats);
+                (uint32_t)p, (uint32_t)root, (int)(n - 1), plan.skip[k], (int)shift, (int32_t)(j + 1), stats);
         }
     }
     if (q > 0) {
@@ -595,7 +603,8 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
         const int64_t shift = (i / q) * q - plan.x;
         reduce_round_kernel<<<round_blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P,
                                                              value_dev, once, twice, (size_t)plan.P, (uint32_t)p,
-                                                             (uint32_t)root, n, plan.skip[k], shift, stats);
+                                                             (uint32_t)root, (int)(n - 1), plan.skip[k], (int)shift,
+                                                             stats);
     }
     for (int64_t b0 = 0; b0 < n; b0 += 65535) {
         const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
