@@ -478,10 +478,11 @@ template <int Q, class Row>
 __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const uint32_t *low_frame,
                                                   uint32_t u_low, int j_high, uint32_t ahead, uint32_t run_end,
                                                   Row recv_row, Row send_row, uint32_t &recv_flags,
-                                                  uint32_t &send_flags)
+                                                  uint32_t &send_flags, bool any_recv)
 {
     constexpr uint32_t kLowMask = (1u << kLowFrameRounds) - 1u;
-    {   // receive entries: straight-line, a predicated byte store per round
+    if (any_recv) {                                        // the same for the whole warp
+        // receive entries: straight-line, a predicated byte store per round
         uint32_t v03, v47;
         const uint32_t have = low_frame_values<Q>(low_frame[u_low], j_high, v03, v47);
         const uint32_t take = recv_flags & have & kLowMask;
@@ -583,9 +584,10 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
                 for (int i = 1; i < kMaxRuns; ++i) run += (int)ahead >= runs.start[i] ? 1 : 0;
                 const uint32_t u_low = (uint32_t)runs.state[run].rp + (ahead - (uint32_t)runs.start[run]);
                 const int j_high = runs.state[run].j;      // lowest digit at the shared levels (Q: none)
+                const bool any_recv = __any_sync(0xffffffffu, (recv_flags & kLowMask) != 0u);
                 if (j_high < Q)
                     low_frame_lookups<Q>(tab, low_frame, u_low, j_high, ahead, (uint32_t)runs.start[run + 1],
-                                         recv_row, send_row, recv_flags, send_flags);
+                                         recv_row, send_row, recv_flags, send_flags, any_recv);
             }
             // entries of the high levels that the description left undecided (at most 32, one per
             // lane); each warp takes those of its own rows, once their placeholders are written
