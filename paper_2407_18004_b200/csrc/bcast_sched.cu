@@ -332,17 +332,18 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     const int shape = choose_shape(tab, p, q, descending, shift_x);
     // up to kWarpsPerBlock consecutive tiles per block, fewer while the grid would have less than
     // kBlocksPerSmWanted blocks per SM (short launches want many small blocks).  A block that first
-    // tabulates the search's low states takes more tiles to spread that cost: up to kLowFrameTiles,
-    // aiming at four waves of resident blocks.
+    // tabulates the search's low states takes more tiles to spread that cost: up to kLowFrameTiles.
     int64_t tiles_per_block = n_tiles / ((int64_t)sms * kBlocksPerSmWanted);
     if (tiles_per_block < 1) tiles_per_block = 1;
     if (tiles_per_block > kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
     if (shape == kShapeWarpsLowFrame) {
-        tiles_per_block = n_tiles / ((int64_t)sms * kTableBlocksPerSm * 4);
-        // measured: 4 tiles at p = 2^20+1 (one wave of blocks), 8 at 2^22+1, 16-32 at 2^24+3, 64-128 at 1.2e8
-        const int least = n_tiles < (int64_t)sms * kTableBlocksPerSm * kWarpsPerBlock ? kWarpsPerBlock / 2 : kWarpsPerBlock;
-        if (tiles_per_block < least) tiles_per_block = least;
+        // one wave of resident blocks while that keeps a block within kLowFrameTiles tiles (measured best
+        // from p = 2^20+1 to 2^24+3), else blocks of kLowFrameTiles (p = 1.2e8: 64 or 128 tiles alike,
+        // fewer is slower)
+        const int64_t slots = (int64_t)sms * kTableBlocksPerSm;
+        tiles_per_block = (n_tiles + slots - 1) / slots;
         if (tiles_per_block > kLowFrameTiles) tiles_per_block = kLowFrameTiles;
+        if (tiles_per_block < kWarpsPerBlock / 2) tiles_per_block = kWarpsPerBlock / 2;
     }
     const int grid = (int)((n_tiles + tiles_per_block - 1) / tiles_per_block);
     const int recv_vec = ((uintptr_t)recv_dev & 15u) == 0, send_vec = ((uintptr_t)send_dev & 15u) == 0;
