@@ -433,6 +433,10 @@ static __device__ __forceinline__ void rows_by_search(uint32_t p, uint32_t ancho
     }
 }
 
+// Whether the search completed all kLowFrameRounds rounds of the word inside the low levels; round
+// kLowFrameRounds is then the lowest shared digit, like a kLowFramePop nibble.
+__device__ __forceinline__ bool low_frame_full(uint32_t word) { return (word >> 28) < kLowFramePop; }
+
 // Search for one deferred item; emit(table, row, k, value) receives every wanted entry
 // (table 0 = receive, 1 = send; row relative to the group's first row).
 template <class Emit>
@@ -467,7 +471,10 @@ __device__ __forceinline__ uint32_t low_frame_values(uint32_t word, int j_high, 
     rounds_4_7 = add_bytes(hi, kMinusQ);
     // one bit per byte: 0x80 of each byte gathered into bits 0..3
     const uint32_t have_lo = ~none_lo & 0x80808080u, have_hi = ~none_hi & 0x80808080u;
-    return ((have_lo * 0x00204081u) >> 28) | (((have_hi * 0x00204081u) >> 28) << 4);
+    uint32_t have = ((have_lo * 0x00204081u) >> 28) | (((have_hi * 0x00204081u) >> 28) << 4);
+    // eight rounds inside the low levels use up every index there, so the ninth is the return past them
+    if (low_frame_full(word)) have |= 1u << kLowFrameRounds;
+    return have;
 }
 
 // Undecided low rounds from the table of the search's low states (low_frame_entry): the
@@ -480,7 +487,7 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
                                                   Row recv_row, Row send_row, uint32_t &recv_flags,
                                                   uint32_t &send_flags, bool any_recv)
 {
-    constexpr uint32_t kLowMask = (1u << kLowFrameRounds) - 1u;
+    constexpr uint32_t kLowMask = (2u << kLowFrameRounds) - 1u;   // the table's rounds and the one after them
     if (any_recv) {                                        // the same for the whole warp
         // receive entries: straight-line, a predicated byte store per round
         uint32_t v03, v47;
@@ -489,6 +496,7 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
 #pragma unroll
         for (int k = 0; k < kLowFrameRounds && k < Q; ++k)
             if ((take >> k) & 1u) recv_row(k, (int)(int8_t)((k < 4 ? v03 : v47) >> (8 * (k & 3))));
+        if (kLowFrameRounds < Q && ((take >> kLowFrameRounds) & 1u)) recv_row(kLowFrameRounds, j_high - Q);
         recv_flags ^= take;
     }
     // send entries: at most four per rank (Theorem 3), one table word each
@@ -498,7 +506,9 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
         todo &= todo - 1u;
         const uint32_t skip_k = skip_of(make_geometry(tab.skip[Q]), k);
         if (ahead + skip_k < run_end) {
-            const uint32_t nib = (low_frame[u_low + skip_k] >> (4 * k)) & 15u;
+            const uint32_t word_t = low_frame[u_low + skip_k];
+            const uint32_t nib = k < kLowFrameRounds ? (word_t >> (4 * k)) & 15u
+                                                     : (low_frame_full(word_t) ? kLowFramePop : kLowFrameNone);
             if (nib <= kLowFramePop) {
                 send_row(k, (nib == kLowFramePop ? j_high : (int)nib) - Q);
                 send_flags ^= 1u << k;
@@ -575,7 +585,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
             auto st = apply_tile_runs<Q>(runs, (int)ahead, recv_row, send_row);
             closed_form_levels<Q, kSharedFrom>(tab, st, recv_row, send_row, recv_flags, send_flags);
             closed_form_finish<Q>(tab, r, st.j, recv_row, send_row, recv_flags);
-            constexpr uint32_t kLowMask = (1u << kLowFrameRounds) - 1u;
+            constexpr uint32_t kLowMask = (2u << kLowFrameRounds) - 1u;
             if (low_frame != nullptr && __any_sync(0xffffffffu, ((recv_flags | send_flags) & kLowMask) != 0u)) {
                 // the rank's state below the shared levels, read again from its run's description
                 // rather than kept in registers across the pass
