@@ -186,7 +186,10 @@ __device__ __forceinline__ uint32_t closed_form_rows(const LevelTables &tab, uin
 //          evaluated inside the suspicious intervals (rare) and undecided entries are noted
 //          in the tile's pending list.
 constexpr int kSharedFrom = 9;
-constexpr int kMaxRuns = 4;
+// A run is as long as there are values of the remainder below kSharedFrom for its digits: at least
+// skip[kSharedFrom] - 1 >= 2^(kSharedFrom-1) = kThreads ranks, so a tile of kThreads rows meets at most one
+// boundary between runs.  (A tile that would need more is given up and walked rank by rank.)
+constexpr int kMaxRuns = 2;
 constexpr int kMaxPending = 32;
 constexpr int kSharedLevels = 31 - kSharedFrom;         // most levels a description can hold
 

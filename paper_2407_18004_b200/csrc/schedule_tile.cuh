@@ -363,9 +363,11 @@ struct SharedTile {
 // The launch shapes of bcast_schedule proper.  After the run descriptions are built no warp
 // waits for another: each takes its own 32 rows of every tile through the closed-form pass
 // and streams them out at once, undecided entries included (with whatever the pass left
-// there).  What is undecided is queued per group of kWarpsPerBlock tiles, and when the
-// group's tiles are out the whole block works the queues off, storing every entry straight
-// into the output table, over the placeholder:
+// there).  What is undecided is queued, and between two groups of kWarpsPerBlock tiles the whole
+// block works the queues off, storing every entry straight into the output table, over the
+// placeholder -- after every group where the block's first group fills a sixth of a queue (a
+// dirty p), else once a queue is a third full and after the last group (a p with few undecided
+// entries gathers several groups' worth, which keeps more lanes busy per search):
 //   1. searches (DeferredItem): the receive schedule of a virtual rank is searched up to a round k;
 //      kind 0 writes the receive entries of the rank's own row for every round up to k (the search
 //      yields them all, and those the pass had decided are the same), kind 1 the send entry of
@@ -377,12 +379,12 @@ struct SharedTile {
 // per warp even fewer.)
 struct DeferredItem {
     uint32_t rank;                                         // virtual rank whose receive schedule is searched
-    uint32_t what;                                         // output row relative to the group | k << 11 | kind << 16
+    uint32_t what;                                         // output row relative to the block | k << 14 | kind << 19
 };                                                         // kind 0: every round up to k; kind 1: round k alone
 
 constexpr int kDeferredCapacity = 384;
-constexpr int kFixupCapacity = 1024;
-constexpr int kGroupRows = kWarpsPerBlock * kThreads;  // rows of a group of tiles: fix-ups hold a row in 11 bits
+constexpr int kFixupCapacity = 768;
+constexpr int kGroupRows = kWarpsPerBlock * kThreads;  // rows of a group of tiles
 constexpr int kLowFrameTiles = 64;                     // most tiles of a block that builds the table of low states
 constexpr int kLowFrameStates = 512;                   // skip[kSharedFrom] <= 2^kSharedFrom states of the low frame
 
@@ -396,11 +398,11 @@ constexpr int kDescWarpsFromQ = 16;                    // smallest q with a desc
 
 struct DeferredQueue {
     DeferredItem items[kDeferredCapacity];
-    uint16_t fixups[kFixupCapacity];                       // row relative to the group | k << 11
+    uint32_t fixups[kFixupCapacity];                       // row relative to the block | k << 14
     uint32_t low_frame[kLowFrameStates];                   // low_frame_entry(u) for u < skip[kSharedFrom], if built
     uint32_t need_recv[kWarpsPerBlock][32];                // per warp and row of its slice: rounds to search
-    int n_items[2];                                        // counters for groups of tiles taken in turn
-    int n_fixups[2];
+    int n_items;
+    int n_fixups;
     uint32_t overflow;                                     // groups of the block (a bit each) that found a queue full
 };
 
@@ -442,9 +444,9 @@ __device__ __forceinline__ bool low_frame_full(uint32_t word) { return (word >> 
 template <class Emit>
 __device__ __forceinline__ void resolve_deferred(const Geometry &g, const DeferredItem &it, Emit emit)
 {
-    const uint32_t row = it.what & 2047u;
-    const int k_last = (int)((it.what >> 11) & 31u);
-    const bool one_send = (it.what >> 16) != 0u;
+    const uint32_t row = it.what & 16383u;
+    const int k_last = (int)((it.what >> 14) & 31u);
+    const bool one_send = (it.what >> 19) != 0u;
     NoStats ns;
     recv_search_fast(g, it.rank, k_last, [&](int k, int val) {
         if (!one_send) emit(0, row, k, val);
@@ -525,11 +527,14 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
 template <int Q, bool desc, class Tile>
 __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry &g,
                                           const TileRuns<typename WalkInt<Q>::type> &runs,
-                                          uint32_t r_first, uint32_t rows, uint32_t group_row0,
+                                          uint32_t r_first, uint32_t rows, uint32_t block_row0,
                                           uint32_t group_rows, const Tile &tile,
-                                          bool want_recv, bool want_send, DeferredQueue &dq, int phase,
+                                          bool want_recv, bool want_send, DeferredQueue &dq,
                                           uint32_t group_bit, int capacity_cut, const uint32_t *low_frame)
 {
+    // block_row0: the tile's first output row relative to the block's; groups are kGroupRows rows each,
+    // so its place within its group is the remainder
+    const uint32_t group_row0 = block_row0 & (uint32_t)(kGroupRows - 1);
     // index: the thread's row of the staged tile = its output row within the tile.  The ranks of a tile
     // ascend with the row, or descend (Algorithm 7's tables); `ahead` is the thread's place counted from
     // the tile's lowest rank r_first, which is how the run descriptions number the rows.
@@ -550,7 +555,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     __syncwarp();
 
     auto defer = [&](const DeferredItem &it) {
-        const int slot = atomicAdd(&dq.n_items[phase], 1);
+        const int slot = atomicAdd(&dq.n_items, 1);
         if (slot < kDeferredCapacity - capacity_cut) {
             dq.items[slot] = it;
         } else {
@@ -566,15 +571,15 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
         const uint32_t out_row = group_row0 + row;
         const bool in_group = desc ? out_row >= skip_k : out_row + skip_k < group_rows;
         if (want_recv && in_group) {
-            const int slot = atomicAdd(&dq.n_fixups[phase], 1);
+            const int slot = atomicAdd(&dq.n_fixups, 1);
             if (slot < kFixupCapacity - capacity_cut * (kFixupCapacity / kDeferredCapacity)) {
-                dq.fixups[slot] = (uint16_t)(out_row | ((uint32_t)k << 11));
+                dq.fixups[slot] = (block_row0 + row) | ((uint32_t)k << 14);
                 return;
             }
         }
         uint32_t t = rr + skip_k;
         if (t >= g.p) t -= g.p;
-        defer(DeferredItem{t, out_row | ((uint32_t)k << 11) | (1u << 16)});
+        defer(DeferredItem{t, (block_row0 + row) | ((uint32_t)k << 14) | (1u << 19)});
     };
 
     uint32_t recv_flags = 0, send_flags = 0;
@@ -635,7 +640,7 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
     }
     __syncwarp();
     const uint32_t mine = (want_recv ? recv_flags : 0u) | need_recv[lane];
-    if (mine != 0u) defer(DeferredItem{r, (group_row0 + index) | ((uint32_t)(31 - __clz(mine)) << 11)});
+    if (mine != 0u) defer(DeferredItem{r, (block_row0 + index) | ((uint32_t)(31 - __clz(mine)) << 14)});
 }
 
 }  // namespace bcast

@@ -66,7 +66,7 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
     if (kDescWarps || shape != kShapeBlockPerTile) {       // host: never with the shifted rows
         constexpr bool desc = kDescWarps;
         DeferredQueue &dq = queues.deferred;
-        if (threadIdx.x < 2) { dq.n_items[threadIdx.x] = 0; dq.n_fixups[threadIdx.x] = 0; }
+        if (threadIdx.x == 0) { dq.n_items = 0; dq.n_fixups = 0; }
         if (threadIdx.x == 2) dq.overflow = 0u;
         // the low rounds of the search for every low state of this p, when the host expects
         // enough undecided entries to pay for it
@@ -78,22 +78,26 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
                 low_frame = dq.low_frame;
             }
         }
-        for (int done = 0, phase = 0; done < tiles_per_block; done += kWarpsPerBlock, phase ^= 1) {
+        const size_t block_base = (size_t)block_first_tile * kThreads * (size_t)Q;
+        const int item_room = kDeferredCapacity - capacity_cut;
+        const int fixup_room = kFixupCapacity - capacity_cut * (kFixupCapacity / kDeferredCapacity);
+        bool gather = false;                               // whether later groups may share a drain
+        for (int done = 0; done < tiles_per_block; done += kWarpsPerBlock) {
             const uint32_t group = block_first_tile + (uint32_t)done;
             if (group >= n_tiles) break;
             const int n_slots = min(kWarpsPerBlock, tiles_per_block - done);
             const uint32_t group_rows = min((uint32_t)n_slots * kThreads, n_ranks - group * kThreads);
             describe_group(group, n_slots);
-            __syncthreads();                               // descriptions (and table) built, this phase's queues empty
+            __syncthreads();                               // descriptions (and table) built, queues reset if drained
             for (int slot = 0; slot < n_slots; ++slot) {
                 const uint32_t t = group + (uint32_t)slot;
                 if (t >= n_tiles) break;
                 const uint32_t first = t * kThreads;
                 const uint32_t rows = min((uint32_t)kThreads, n_ranks - first);
                 const SharedTile<Q> tile{recv_bytes, send_bytes, rows, false};
-                warp_pass<Q, desc>(tab, g, runs[slot], first_rank_of(first, rows), rows, (uint32_t)slot * kThreads,
-                                   group_rows, tile, want_recv, want_send, dq, phase, 1u << (done / kWarpsPerBlock),
-                                   capacity_cut, low_frame);
+                warp_pass<Q, desc>(tab, g, runs[slot], first_rank_of(first, rows), rows,
+                                   (uint32_t)(done + slot) * kThreads, group_rows, tile, want_recv, want_send, dq,
+                                   1u << (done / kWarpsPerBlock), capacity_cut, low_frame);
                 __syncwarp();                              // the slice is staged
                 const uint32_t my_first = (uint32_t)warp * 32u;
                 if (my_first < rows) {
@@ -105,30 +109,33 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
                 }
                 __syncwarp();                              // flushed before the next tile's pass overwrites it
             }
-            __syncthreads();                               // every slice of the group is out; now its searches
-            const size_t group_base = (size_t)group * kThreads * (size_t)Q;
-            const int n_items = min(dq.n_items[phase], kDeferredCapacity - capacity_cut);
-            const int n_fixups = min(dq.n_fixups[phase],
-                                     kFixupCapacity - capacity_cut * (kFixupCapacity / kDeferredCapacity));
+            __syncthreads();                               // every slice of the group is out
+            // Work the queues off now?  The same answer in every thread: the counters rest until the next pass.
+            // The block's first group tells how dense the undecided entries of this p are.
+            const bool last = done + kWarpsPerBlock >= tiles_per_block || group + kWarpsPerBlock >= n_tiles;
+            const int queued_items = dq.n_items, queued_fixups = dq.n_fixups;
+            if (done == 0) gather = queued_items <= item_room / 6 && queued_fixups <= fixup_room / 6;
+            if (!last && gather && queued_items <= item_room / 3 && queued_fixups <= fixup_room / 3) continue;
+            const int n_items = min(queued_items, item_room);
+            const int n_fixups = min(queued_fixups, fixup_room);
             for (int i = threadIdx.x; i < n_items; i += kThreads) {
                 resolve_deferred(g, dq.items[i], [&](int table, uint32_t row, int k, int val) {
                     int32_t *out = table == 0 ? recv_out : send_out;
-                    out[group_base + (size_t)row * Q + k] = val;
+                    out[block_base + (size_t)row * Q + k] = val;
                 });
             }
-            if (n_fixups > 0) {                            // the same for the whole block
-                __syncthreads();                           // the group's receive entries are final in the table
-                for (int i = threadIdx.x; i < n_fixups; i += kThreads) {
-                    const uint32_t f = dq.fixups[i];
-                    const uint32_t row = f & 2047u, k = f >> 11;
-                    const uint32_t from = desc ? row - tab.skip[k] : row + tab.skip[k];
-                    send_out[group_base + (size_t)row * Q + k] = __ldcg(recv_out + group_base + (size_t)from * Q + k);
-                }
+            if (n_fixups > 0) __syncthreads();             // the receive entries of every group so far are final
+            for (int i = threadIdx.x; i < n_fixups; i += kThreads) {
+                const uint32_t f = dq.fixups[i];
+                const uint32_t row = f & 16383u, k = f >> 14;
+                const uint32_t from = desc ? row - tab.skip[k] : row + tab.skip[k];
+                send_out[block_base + (size_t)row * Q + k] = __ldcg(recv_out + block_base + (size_t)from * Q + k);
             }
-            // the other phase's counters were last read in the previous group's drain, which every
-            // thread had left before this group's passes began
-            if (threadIdx.x < 2) {
-                if (threadIdx.x == 0) dq.n_items[phase ^ 1] = 0; else dq.n_fixups[phase ^ 1] = 0;
+            // (every thread read the counters before its first search; the next pushes come after the barrier
+            // that follows the next group's descriptions)
+            if (queued_items + queued_fixups > 0) {
+                __syncthreads();
+                if (threadIdx.x == 0) { dq.n_items = 0; dq.n_fixups = 0; }
             }
         }
         // groups that found a queue full (bit = number of the group within the block): their rows
