@@ -365,8 +365,8 @@ struct SharedTile {
 // and streams them out at once, undecided entries included (with whatever the pass left
 // there).  What is undecided is queued, and between two groups of kWarpsPerBlock tiles the whole
 // block works the queues off, storing every entry straight into the output table, over the
-// placeholder -- after every group where the block's first group fills a sixth of a queue (a
-// dirty p), else once a queue is a third full and after the last group (a p with few undecided
+// placeholder -- after every group where the block's first group fills a quarter of a queue (a
+// dirty p), else once a queue is half full and after the last group (a p with few undecided
 // entries gathers several groups' worth, which keeps more lanes busy per search):
 //   1. searches (DeferredItem): the receive schedule of a virtual rank is searched up to a round k;
 //      kind 0 writes the receive entries of the rank's own row for every round up to k (the search

@@ -114,8 +114,8 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
             // The block's first group tells how dense the undecided entries of this p are.
             const bool last = done + kWarpsPerBlock >= tiles_per_block || group + kWarpsPerBlock >= n_tiles;
             const int queued_items = dq.n_items, queued_fixups = dq.n_fixups;
-            if (done == 0) gather = queued_items <= item_room / 6 && queued_fixups <= fixup_room / 6;
-            if (!last && gather && queued_items <= item_room / 3 && queued_fixups <= fixup_room / 3) continue;
+            if (done == 0) gather = queued_items <= item_room / 4 && queued_fixups <= fixup_room / 4;
+            if (!last && gather && queued_items <= item_room / 2 && queued_fixups <= fixup_room / 2) continue;
             const int n_items = min(queued_items, item_room);
             const int n_fixups = min(queued_fixups, fixup_room);
             for (int i = threadIdx.x; i < n_items; i += kThreads) {
