@@ -58,24 +58,32 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s: MEASURED_PEAKS.json is absent)"
 
 
-def kernel_source_hash() -> str:
-    """sha256 over the CUDA sources: a recorded DRAM-traffic figure is only quoted for the kernel it was taken on."""
-    import glob
+KERNEL_SOURCES = {
+    "schedule_table_kernel": ("schedule_core.cuh", "schedule_fast.cuh", "schedule_tile.cuh", "table_kernel.cuh",
+                              "table_q_low.cu", "table_q_mid.cu", "table_q_high.cu", "table_q_top.cu", "bcast_sched.cu"),
+    "schedule_batch_kernel": ("schedule_core.cuh", "schedule_fast.cuh", "schedule_tile.cuh", "bcast_sched.cu"),
+    "verify_sweep_kernel": ("schedule_core.cuh", "schedule_fast.cuh", "schedule_tile.cuh", "bcast_sweep.cu"),
+}
+
+
+def kernel_source_hash(kernel: str) -> str:
+    """sha256 over the CUDA sources a kernel is compiled from: a recorded counter is only quoted for the kernel it
+    was taken on."""
     import hashlib
     h = hashlib.sha256()
-    for path in sorted(glob.glob(os.path.join(ROOT, "paper_2407_18004_b200", "csrc", "*"))):
-        with open(path, "rb") as fh:
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, "paper_2407_18004_b200", "csrc", name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()
 
 
 def recorded_counters(kernel: str, key: str):
-    """A line `kernel key sha256-of-csrc a b` of profiles/counters.txt as (a, b), or None when there is none for
+    """A line `kernel key sha256-of-its-sources a b` of profiles/counters.txt as (a, b), or None when there is none for
     the sources as they are now (ncu counters of a small stand-in launch; see the file for what a and b are)."""
     path = os.path.join(ROOT, "profiles", "counters.txt")
     if not os.path.exists(path):
         return None
-    sha = kernel_source_hash()
+    sha = kernel_source_hash(kernel)
     with open(path) as fh:
         for line in fh:
             parts = line.split()
@@ -629,6 +637,11 @@ def build_other(args, torch, bs):
     q = bs.bcast_q(p)
     n = args.blocks
     rounds = n - 1 + q
+    bs.bcast_set_simulate_rounds({"auto": bs.BCAST_ROUNDS_AUTO, "launches": bs.BCAST_ROUNDS_LAUNCHES,
+                                  "fused": bs.BCAST_ROUNDS_FUSED}[args.rounds])
+    fused = args.rounds != "launches"
+    round_launches = (rounds + 65535) // 65536 + 1 if fused else rounds     # fused: up to 65536 rounds a launch, and the seal
+    form = "all rounds in cooperative launches" if fused else "one launch per round"
     recv = torch.empty((p, q), dtype=torch.int32, device="cuda")
     send = torch.empty((p, q), dtype=torch.int32, device="cuda")
     bs.bcast_schedule(p, 0, 0, p, recv, send, stream)
@@ -660,9 +673,10 @@ def build_other(args, torch, bs):
         # tables turned into bytes (8q read, 2q written per processor), arrival table set and counted (4 B per
         # cell each), and per round and processor two table bytes, two arrival reads and one arrival write
         nbytes = p * (10 * q + 8 * n + rounds * 14)
-        return dict(label="Algorithm 1 by all processors of p=%d (q=%d), n=%d blocks, %d rounds, tables on the device"
-                          % (p, q, n, rounds), metric="simulated_block_deliveries_per_s", unit="blocks/s",
-                    units=(p - 1) * n, bytes=nbytes, step=step, launches=rounds + 3, kernel="broadcast_round_kernel",
+        return dict(label="Algorithm 1 by all processors of p=%d (q=%d), n=%d blocks, %d rounds (%s), tables on the device"
+                          % (p, q, n, rounds, form), metric="simulated_block_deliveries_per_s", unit="blocks/s",
+                    units=(p - 1) * n, bytes=nbytes, step=step, launches=round_launches + 4,
+                    kernel="broadcast_rounds_kernel" if fused else "broadcast_round_kernel",
                     bound="hbm", e2e=e2e_step, h2d=0, d2h=64, oracle=oracle_sample,
                     extra=lambda: {"stats": stats.tolist()})
     gen = torch.Generator(device="cuda")
@@ -698,9 +712,10 @@ def build_other(args, torch, bs):
     # round and processor: three table bytes, the sender's value read, the own value read and written, sent
     # count read twice and written once
     nbytes = p * (10 * q + 18 * n + rounds * (3 + 8 + 16 + 3))
-    return dict(label="Observation 1.3's reduction by all processors of p=%d (q=%d), n=%d blocks, %d rounds"
-                      % (p, q, n, rounds), metric="simulated_partial_results_per_s", unit="blocks/s",
-                units=(p - 1) * n, bytes=nbytes, step=step, launches=rounds + 4, kernel="reduce_round_kernel",
+    return dict(label="Observation 1.3's reduction by all processors of p=%d (q=%d), n=%d blocks, %d rounds (%s)"
+                      % (p, q, n, rounds, form), metric="simulated_partial_results_per_s", unit="blocks/s",
+                units=(p - 1) * n, bytes=nbytes, step=step, launches=round_launches + 2,
+                kernel="reduce_rounds_kernel" if fused else "reduce_round_kernel",
                 bound="hbm", e2e=e2e_step, h2d=0, d2h=64 + 8 * n, oracle=oracle_sample,
                 extra=lambda: {"stats": stats.tolist()})
 
@@ -778,7 +793,7 @@ def run_other(args):
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None, "peak_source": peak_src,
                     "kernel": wl["kernel"], "bytes_per_step": wl["bytes"],
-                    "note": "algorithmic bytes of the whole step over the step's time (many short launches)"}
+                    "note": "algorithmic bytes of the whole step over the step's time (all of its launches)"}
     else:
         # bound by instruction issue: warp instructions of one launch (recorded from ncu while the sources
         # are unchanged) over its time, against one instruction per scheduler and clock
@@ -899,6 +914,9 @@ def main():
                          "sweep: fused verification of every p in [2, 65536]; simulate / reduce: Algorithm 1 and "
                          "its reversal run by all processors of --workload (default p=2^20+1) with --blocks blocks")
     ap.add_argument("--blocks", type=int, default=64, help="n, the number of blocks (shifted, simulate, reduce)")
+    ap.add_argument("--rounds", default="auto", choices=["auto", "launches", "fused"],
+                    help="simulate / reduce: one kernel launch per communication round, or all rounds in "
+                         "cooperative launches (auto: fused where the device has them)")
     ap.add_argument("--queries", type=int, default=2 ** 24, help="number of queries (batch)")
     ap.add_argument("--sweep-lo", type=int, default=2, help="first p of the sweep")
     ap.add_argument("--sweep-hi", type=int, default=65536, help="last p of the sweep")

@@ -11,9 +11,10 @@
  *  - Plain C types only.  "host" pointers are ordinary process memory; "device"
  *    pointers are CUDA global memory of the current device.  The caller owns
  *    every buffer and the library allocates nothing.  It is thread-safe and
- *    keeps no state between calls, with two documented exceptions: the
- *    process-wide launch-shape override (bcast_set_launch_shape) and the
- *    built-in scratch array of bcast_verify_sweep_static.
+ *    keeps no state between calls, with three documented exceptions: the
+ *    process-wide overrides of bcast_set_launch_shape and
+ *    bcast_set_simulate_rounds, and the built-in scratch array of
+ *    bcast_verify_sweep_static.
  *  - cuda_stream is a cudaStream_t passed as void* (NULL = default stream).
  *    Device work is enqueued on it and the call returns without synchronising.
  *  - Return value: >= 0 on success (where stated, the value of q), otherwise a
@@ -67,6 +68,11 @@ extern "C" {
 #define BCAST_SHAPE_LOWFRAME   2        /* the same, low rounds looked up in a per-block table     */
 #define BCAST_SHAPE_WARPS_TIGHT 3       /* BCAST_SHAPE_WARPS with next to no queue space: for tests */
                                         /* of the path that recomputes a group whose queues ran full */
+
+/* How bcast_simulate_broadcast / bcast_simulate_reduce launch their rounds (bcast_set_simulate_rounds). */
+#define BCAST_ROUNDS_AUTO      0        /* fused where the device has cooperative launches (default) */
+#define BCAST_ROUNDS_LAUNCHES  1        /* one kernel launch per communication round                  */
+#define BCAST_ROUNDS_FUSED     2        /* all rounds in cooperative launches, blocks meet per round   */
 
 #define BCAST_STATIC_SWEEP_BYTES  (8u << 20)   /* built-in scratch of bcast_verify_sweep_static */
 #define BCAST_STATIC_SWEEP_MAX_P  65536        /* largest p_hi it accepts                       */
@@ -271,10 +277,31 @@ int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev
  * bcast_simulate_scratch_bytes(p, n, 0) bytes; it receives round-major byte
  * copies of the tables and a bit per (processor, block) for who holds what.
  * Contents after the call are unspecified.
- * Launches n-1+q small kernels on cuda_stream, asynchronously.  Returns q.
+ * Asynchronous on cuda_stream.  Returns q.
  * Limits: n < 2^31 - 64; n * p int32 cells must fit the caller's memory.
+ *
+ * The n-1+q rounds run either as one small launch each or, by default where the
+ * device has cooperative launches, inside cooperative launches of up to 65536
+ * rounds whose blocks meet at a counter in the scratch between two rounds (a
+ * round of 2^20 processors is too short to pay for a launch of its own).  That
+ * wait is bounded: should a block see no progress for about two seconds (all
+ * blocks of a cooperative launch are resident, so this is not expected), every
+ * block stops and ALL EIGHT statistics words are set to UINT64_MAX; arrival_dev
+ * is then unspecified.  Both forms give the same arrival table and statistics.
  */
 int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction);
+
+/*
+ * Not from the paper: forces how the two single-root simulators launch their
+ * rounds from now on, process-wide (tuning, and tests that run both forms on the
+ * same tables): one of BCAST_ROUNDS_*.  BCAST_ROUNDS_FUSED on a device without
+ * cooperative launches makes those calls return BCAST_ECUDA.  The environment
+ * variable BCAST_SIMULATE_ROUNDS=launches|fused, read once at the first
+ * simulation, does the same until this is called.  Host only.  Returns BCAST_OK
+ * or BCAST_EINVAL_SHAPE.
+ */
+int bcast_set_simulate_rounds(int mode);
+
 int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
                              const int32_t *recvblock_dev, const int32_t *sendblock_dev,
                              int32_t *arrival_dev, uint64_t *stats_dev,
@@ -308,8 +335,9 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
  *   [6] partial results combined            (correct tables: (p-1)*n)
  *   [7] unused, 0
  * scratch_dev: at least bcast_simulate_scratch_bytes(p, n, 1) bytes, 16-byte
- * aligned.  Tables, limits, asynchrony and return value as for
- * bcast_simulate_broadcast.
+ * aligned.  Tables, limits, asynchrony, the two ways of launching the rounds
+ * (statistics all UINT64_MAX if the bounded wait ran out; value_dev and
+ * result_dev then unspecified) and return value as for bcast_simulate_broadcast.
  */
 int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
                           const int32_t *recvblock_dev, const int32_t *sendblock_dev,

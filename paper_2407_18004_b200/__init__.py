@@ -20,6 +20,7 @@ BCAST_MAX_Q = 31
 BCAST_STATIC_SWEEP_MAX_P = 65536
 BCAST_UNRESOLVED = -128
 BCAST_SHAPE_AUTO, BCAST_SHAPE_BLOCK, BCAST_SHAPE_WARPS, BCAST_SHAPE_LOWFRAME, BCAST_SHAPE_WARPS_TIGHT = -1, 0, 1, 2, 3
+BCAST_ROUNDS_AUTO, BCAST_ROUNDS_LAUNCHES, BCAST_ROUNDS_FUSED = 0, 1, 2
 
 _lib = None
 
@@ -40,6 +41,7 @@ def _load():
         lib.bcast_strerror.restype = ctypes.c_char_p
         lib.bcast_q.argtypes = [i32]
         lib.bcast_set_launch_shape.argtypes = [ctypes.c_int]
+        lib.bcast_set_simulate_rounds.argtypes = [ctypes.c_int]
         lib.bcast_skips.argtypes = [i32, vp]
         lib.bcast_schedule.argtypes = [i32, i32, i64, i64, vp, vp, vp]
         lib.bcast_schedule_host.argtypes = [i32, i32, i64, i64, vp, vp, vp, i64, vp]
@@ -100,6 +102,10 @@ def bcast_strerror(code: int) -> str:
 
 def bcast_set_launch_shape(shape: int) -> int:
     return _check(_load().bcast_set_launch_shape(shape))
+
+
+def bcast_set_simulate_rounds(mode: int) -> int:
+    return _check(_load().bcast_set_simulate_rounds(mode))
 
 
 def bcast_q(p: int) -> int:

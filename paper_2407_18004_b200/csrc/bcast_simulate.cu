@@ -24,6 +24,10 @@
 //     64-bit statistics with one atomic per block and counter that is not zero.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <atomic>
 
 #include "../../include/bcast_sched.h"
 
@@ -98,12 +102,18 @@ transpose_tables_kernel(const int32_t *__restrict__ recv_tab, const int32_t *__r
     const int n_entries = (int)rows * q;
     const int32_t *src = in + (size_t)first * q;
     unsigned int bad = 0;
+    // entry i of the tile is column i mod q of row i / q: kept up to date from one step to the next
+    // (a division per entry would cost more than the load)
+    int row = threadIdx.x / q, col = threadIdx.x - row * q;
+    const int row_step = kThreads / q, col_step = kThreads - row_step * q;
     for (int i = threadIdx.x; i < n_entries; i += kThreads) {
-        const int v = src[i];
+        const int v = __ldcs(src + i);
         const bool ok = v >= -q && v <= q - 1;
         bad += ok ? 0u : 1u;
-        const int row = i / q;
-        tile[row * 33 + (i - row * q)] = ok ? (int8_t)v : kInvalid;
+        tile[row * 33 + col] = ok ? (int8_t)v : kInvalid;
+        row += row_step;
+        col += col_step;
+        if (col >= q) { col -= q; ++row; }
     }
     __syncthreads();
     if (threadIdx.x < rows)
@@ -112,11 +122,12 @@ transpose_tables_kernel(const int32_t *__restrict__ recv_tab, const int32_t *__r
     stats_end(bstats, stats);
 }
 
+// The root's column of the arrival table (the rest is set to -1 by a memset): it holds every block from the start.
 __global__ void __launch_bounds__(kThreads)
-init_arrival_kernel(int32_t *__restrict__ arrival, uint32_t p, uint32_t root)
+root_arrival_kernel(int32_t *__restrict__ arrival, uint32_t p, uint32_t root, int64_t n)
 {
-    const uint32_t a = blockIdx.x * kThreads + threadIdx.x;
-    if (a < p) arrival[(size_t)blockIdx.y * p + a] = a == root ? 0 : -1;
+    const int64_t b = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (b < n) arrival[(size_t)b * p + root] = 0;
 }
 
 // Bit sets over the blocks, a word of 64 blocks per processor: set[w * P + a].  Cleared for everybody
@@ -164,51 +175,211 @@ __device__ __forceinline__ int block32(int8_t entry, int shift, int last)
 // round; the bit can only be about to change in this round if f is itself receiving that very
 // block now, and then the answer is taken from f's arrival cell, which is -1 or >= round for
 // anything not held before, whether or not f's write is seen.
-__global__ void __launch_bounds__(kThreads)
-broadcast_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
-                       int32_t *arrival, unsigned long long *held, size_t P, uint32_t p, uint32_t root,
-                       int last, uint32_t skip_k, int shift, int32_t round, unsigned long long *stats)
-{
-    __shared__ BlockStats bstats;
-    stats_begin(bstats);
+struct RoundCounts {
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
+};
+
+__device__ __forceinline__ void add_round_counts(BlockStats &bs, const RoundCounts &c)
+{
+    add_stat(bs, 0, c.c0);
+    add_stat(bs, 1, c.c1);
+    add_stat(bs, 2, c.c2);
+    add_stat(bs, 3, c.c3);
+    add_stat(bs, 6, c.c6);
+}
+
+// What the rounds of the broadcast need besides the round's own rows of the byte tables.
+struct BroadcastFrame {
+    int32_t *arrival;                      // arrival[b * p + a]: the round in which processor a got block b
+    unsigned long long *held;              // held[w * P + a]: a bit per block of word w that processor a holds
+    size_t P;
+    uint32_t p, root;
+    int last;                              // n - 1
+};
+
+// One communication round of Algorithm 1 for every processor: skip index k (the rows of the
+// byte tables passed in), blocks = entry + shift, `round` counted from 1.
+//
+// Who holds what is kept twice: arrival[b][a], the result, written once per delivery, and
+// held[w][a], a bit per block, which is what the round reads (8 bytes per processor, consecutive
+// processors side by side, where the arrival cells of a round lie in up to 2q different rows).
+// Thread a alone writes a's word.  A reader of f's word asks whether f held the block BEFORE the
+// round; the bit can only be about to change in this round if f is itself expecting that very
+// block now, and then the answer is taken from f's arrival cell, which is -1 or >= round for
+// anything not held before, whether or not f's write is seen.  What another processor wrote is
+// read past L1 (ld.global.cg): in the kernel that runs several rounds in one launch a line that
+// L1 kept from an earlier round would be stale.
+__device__ __forceinline__ void broadcast_round(const BroadcastFrame &fr, const int8_t *__restrict__ recv_k,
+                                                const int8_t *__restrict__ send_k, uint32_t skip_k, int shift,
+                                                int32_t round, RoundCounts &c)
+{
     // a resident grid strides over the processors: a few thousand blocks would each add their
     // counters to the same statistics words, and those atomics would set the pace of the round
-    for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
+    const uint32_t p = fr.p, root = fr.root;
+    for (uint32_t a = blockIdx.x * blockDim.x + threadIdx.x; a < p; a += gridDim.x * blockDim.x) {
         if (a == root) continue;
         const uint32_t f = a >= skip_k ? a - skip_k : a + (p - skip_k);     // from-processor
-        const int want = block32(recv_k[a], shift, last);
+        const int want = block32(recv_k[a], shift, fr.last);
         // f's to-processor is a, which is not the root, so f's send is not suppressed
-        const int sent = block32(send_k[f], shift, last);
+        const int sent = block32(send_k[f], shift, fr.last);
+        // what f itself expects in this round: read here, beside the other two table bytes, not
+        // where it is needed at the end of the chain of loads below
+        const int f_wants = f == root ? -1 : block32(recv_k[f], shift, fr.last);
         if (want < 0) {
-            c3 += sent >= 0 ? 1u : 0u;
+            c.c3 += sent >= 0 ? 1u : 0u;
         } else if (sent != want) {
-            c0 += 1;
+            c.c0 += 1;
         } else {
-            unsigned long long *words = held + (size_t)(want >> 6) * P;
+            unsigned long long *words = fr.held + (size_t)(want >> 6) * fr.P;
             const unsigned long long bit = 1ull << (want & 63);
-            bool f_held = (words[f] & bit) != 0ull;
-            if (f_held && f != root && block32(recv_k[f], shift, last) == want) {
-                const int32_t at_f = arrival[(size_t)want * p + f];          // f may be getting it only now
+            const unsigned long long theirs = __ldcg(words + f), mine = __ldcg(words + a);
+            bool f_held = (theirs & bit) != 0ull;
+            if (f_held && f_wants == want) {
+                const int32_t at_f = __ldcg(fr.arrival + (size_t)want * p + f);    // f may be getting it only now
                 f_held = at_f >= 0 && at_f < round;
             }
-            const unsigned long long mine = words[a];
-            if (!f_held) c1 += 1;                                            // not held before the round
-            else if ((mine & bit) != 0ull) c2 += 1;
+            if (!f_held) c.c1 += 1;                                          // not held before the round
+            else if ((mine & bit) != 0ull) c.c2 += 1;
             else {
                 words[a] = mine | bit;
-                arrival[(size_t)want * p + a] = round;
-                c6 += 1;
+                fr.arrival[(size_t)want * p + a] = round;
+                c.c6 += 1;
             }
         }
     }
-    add_stat(bstats, 0, c0);
-    add_stat(bstats, 1, c1);
-    add_stat(bstats, 2, c2);
-    add_stat(bstats, 3, c3);
-    add_stat(bstats, 6, c6);
-    if (__any_sync(0xffffffffu, c6 != 0u) && (threadIdx.x & 31) == 0) bstats.last_round = (unsigned int)round;
+}
+
+__global__ void __launch_bounds__(kThreads, 8)
+broadcast_round_kernel(const __grid_constant__ BroadcastFrame fr, const int8_t *__restrict__ recv_k,
+                       const int8_t *__restrict__ send_k, uint32_t skip_k, int shift, int32_t round,
+                       unsigned long long *stats)
+{
+    __shared__ BlockStats bstats;
+    stats_begin(bstats);
+    RoundCounts c;
+    broadcast_round(fr, recv_k, send_k, skip_k, shift, round, c);
+    add_round_counts(bstats, c);
+    if (__any_sync(0xffffffffu, c.c6 != 0u) && (threadIdx.x & 31) == 0) bstats.last_round = (unsigned int)round;
     stats_end(bstats, stats);
+}
+
+// ------------------------------------------------------------------ several rounds in one launch
+// The blocks of a cooperative launch (all resident at once, or the launch is refused) meet between
+// two rounds at a counter in the caller's scratch: every block adds one after its threads' writes
+// are fenced, and waits until all blocks of the round have.  The wait is bounded: a block that
+// sees nothing for about two seconds raises `failed`, every block leaves its loop, and the
+// statistics are overwritten with all-ones by seal_stats_kernel.
+struct GridBarrier {
+    unsigned long long arrived;            // blocks that have reached a barrier, over all barriers of the call
+    unsigned int failed;
+};
+static_assert(sizeof(GridBarrier) <= kHeaderBytes, "the barrier lives in the scratch header");
+
+constexpr unsigned int kBarrierSpins = 1u << 23;
+#ifndef BCAST_FUSED_THREADS
+#define BCAST_FUSED_THREADS 1024
+#endif
+#ifndef BCAST_FUSED_BLOCKS
+#define BCAST_FUSED_BLOCKS 2
+#endif
+constexpr int kFusedThreads = BCAST_FUSED_THREADS;     // large blocks: few arrivals per barrier
+constexpr int kFusedBlocks = BCAST_FUSED_BLOCKS;       // resident per SM
+
+// `index` = this barrier's number in the call, from 1.  The arrival is a release (the block's
+// writes, ordered before it by the block barrier, are visible to whoever sees the count) and, for
+// the last block in, an acquire; the others' wait is an acquire.
+__device__ __forceinline__ bool grid_barrier(GridBarrier *gb, unsigned long long index)
+{
+    __shared__ int through;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long target = index * gridDim.x;
+        unsigned long long seen;
+        asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], 1;" : "=l"(seen) : "l"(&gb->arrived) : "memory");
+        bool good = seen + 1ull >= target;
+        for (unsigned int spin = 0; !good && spin < kBarrierSpins; ++spin) {
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(&gb->arrived) : "memory");
+            if (seen >= target) good = true;
+            else if (*(volatile unsigned int *)&gb->failed != 0u) break;
+            else if (spin >= 64u) __nanosleep(200u);
+        }
+        if (!good) *(volatile unsigned int *)&gb->failed = 1u;
+        through = good ? 1 : 0;
+    }
+    __syncthreads();
+    return through != 0;
+}
+
+__global__ void seal_stats_kernel(const GridBarrier *gb, unsigned long long *stats)
+{
+    if (gb->failed != 0u && threadIdx.x < 8) stats[threadIdx.x] = ~0ull;
+}
+
+struct RoundPlan {
+    uint32_t skip[32];
+    int q;
+    int x;
+};
+
+// Counters of a block over many rounds (64 bits: 2^31 rounds of a few thousand processors).
+struct BlockStats64 {
+    unsigned long long count[8];
+    unsigned int last_round;
+};
+
+__device__ __forceinline__ void add_stat64(BlockStats64 &bs, int index, unsigned int mine)
+{
+    const unsigned int total = __reduce_add_sync(0xffffffffu, mine);
+    if (total != 0u && (threadIdx.x & 31) == 0) atomicAdd(&bs.count[index], (unsigned long long)total);
+}
+
+__device__ __forceinline__ void stats64_begin(BlockStats64 &bs)
+{
+    if (threadIdx.x < 8) bs.count[threadIdx.x] = 0ull;
+    if (threadIdx.x == 8) bs.last_round = 0u;
+    __syncthreads();
+}
+
+__device__ __forceinline__ void stats64_end(BlockStats64 &bs, unsigned long long *stats)
+{
+    __syncthreads();
+    if (threadIdx.x < 8 && bs.count[threadIdx.x] != 0ull) atomicAdd(stats + threadIdx.x, bs.count[threadIdx.x]);
+    if (threadIdx.x == 8 && bs.last_round != 0u) atomicMax(stats + 7, (unsigned long long)bs.last_round);
+}
+
+// Rounds j0 .. j1-1 of the broadcast (j counted from 0), one block barrier between two rounds;
+// `barriers_before` = the barriers of the launches before this one in the same call.
+__global__ void __launch_bounds__(kFusedThreads, kFusedBlocks)
+broadcast_rounds_kernel(const __grid_constant__ BroadcastFrame fr, const int8_t *__restrict__ recv_t,
+                        const int8_t *__restrict__ send_t, const __grid_constant__ RoundPlan plan, long long j0, long long j1,
+                        GridBarrier *gb, unsigned long long barriers_before, unsigned long long *stats)
+{
+    __shared__ BlockStats64 bstats;
+    stats64_begin(bstats);
+    const long long i0 = plan.x + j0;
+    int k = (int)(i0 % plan.q);
+    int shift = (int)((i0 / plan.q) * plan.q - plan.x);               // Theorem 1
+    unsigned int last_delivery = 0;
+    unsigned long long barriers = barriers_before;
+    bool failed = false;
+    // a thread's counts of one launch fit 32 bits: at most 65536 rounds of 2^31 / (threads of the grid) processors
+    RoundCounts c;
+    for (long long j = j0; j < j1; ++j) {
+        const unsigned int delivered_before = c.c6;
+        broadcast_round(fr, recv_t + (size_t)k * fr.P, send_t + (size_t)k * fr.P, plan.skip[k], shift, (int32_t)(j + 1), c);
+        if (c.c6 != delivered_before) last_delivery = (unsigned int)(j + 1);
+        if (++k == plan.q) { k = 0; shift += plan.q; }
+        if (j + 1 < j1 && !grid_barrier(gb, ++barriers)) { failed = true; break; }
+    }
+    if (failed) return;
+    add_stat64(bstats, 0, c.c0);
+    add_stat64(bstats, 1, c.c1);
+    add_stat64(bstats, 2, c.c2);
+    add_stat64(bstats, 3, c.c3);
+    add_stat64(bstats, 6, c.c6);
+    last_delivery = __reduce_max_sync(0xffffffffu, last_delivery);
+    if ((threadIdx.x & 31) == 0 && last_delivery != 0u) atomicMax(&bstats.last_round, last_delivery);
+    stats64_end(bstats, stats);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -251,6 +422,49 @@ count_missing_sets_kernel(const unsigned long long *__restrict__ held, size_t P,
 // t sends b in this round, and t adds to value[b][t] only when it receives b and is NOT
 // sending b (a processor that receives the block it is sending would never pass the sum on,
 // which is counted instead); sent[.][a] is read and written by thread a alone.
+__device__ __forceinline__ void reduce_round(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
+                                             uint64_t *value, unsigned long long *once, unsigned long long *twice,
+                                             size_t P, uint32_t p, uint32_t root, int last, uint32_t skip_k,
+                                             int shift, RoundCounts &c)
+{
+    for (uint32_t a = blockIdx.x * blockDim.x + threadIdx.x; a < p; a += gridDim.x * blockDim.x) {
+        uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
+        if (t >= p) t -= p;
+        const int mine = a == root ? -1 : block32(recv_k[a], shift, last);         // what a sends
+        const int got = t == root ? -1 : block32(recv_k[t], shift, last);          // what t sends to a
+        const int want = t == root ? -1 : block32(send_k[a], shift, last);
+        // every load the round may need is issued here, before any of them is looked at: the two
+        // partial results, and a's words of the sets for the block it sends and the block it expects
+        const bool match = want >= 0 && got == want;
+        uint64_t theirs = 0, own = 0;
+        unsigned long long once_mine = 0ull, once_want = 0ull;
+        if (match) {
+            theirs = __ldcg(value + (size_t)want * p + t);                          // t's: read past L1
+            own = value[(size_t)want * p + a];
+            once_want = once[(size_t)(want >> 6) * P + a];
+        }
+        if (mine >= 0) once_mine = once[(size_t)(mine >> 6) * P + a];
+        // how often a has sent a block: bit in once[] after the first time, in twice[] after the second;
+        // thread a alone reads and writes a's words
+        const bool sent_mine = mine >= 0 && ((once_mine >> (mine & 63)) & 1ull) != 0ull;
+        if (sent_mine) c.c2 += 1;
+        if (want < 0) {
+            if (got >= 0) c.c3 += 1;
+        } else if (got != want) {
+            c.c0 += 1;
+        } else if (a != root && (mine == want || ((once_want >> (want & 63)) & 1ull) != 0ull)) {
+            c.c1 += 1;                                     // it would never be passed on
+        } else {
+            value[(size_t)want * p + a] = own + theirs;
+            c.c6 += 1;
+        }
+        if (mine >= 0) {
+            if (sent_mine) twice[(size_t)(mine >> 6) * P + a] |= 1ull << (mine & 63);
+            else once[(size_t)(mine >> 6) * P + a] = once_mine | (1ull << (mine & 63));
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads)
 reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict__ send_k,
                     uint64_t *value, unsigned long long *once, unsigned long long *twice, size_t P,
@@ -259,41 +473,41 @@ reduce_round_kernel(const int8_t *__restrict__ recv_k, const int8_t *__restrict_
 {
     __shared__ BlockStats bstats;
     stats_begin(bstats);
-    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0, c6 = 0;
-    for (uint32_t a = blockIdx.x * kThreads + threadIdx.x; a < p; a += gridDim.x * kThreads) {
-        uint32_t t = a + skip_k;                           // < 2^32: p, skip_k < 2^31
-        if (t >= p) t -= p;
-        const int mine = a == root ? -1 : block32(recv_k[a], shift, last);         // what a sends
-        const int got = t == root ? -1 : block32(recv_k[t], shift, last);          // what t sends to a
-        const int want = t == root ? -1 : block32(send_k[a], shift, last);
-        // how often a has sent a block: bit in once[] after the first time, in twice[] after the second;
-        // thread a alone reads and writes a's words
-        bool sent_mine = false;
-        if (mine >= 0) {
-            sent_mine = (once[(size_t)(mine >> 6) * P + a] >> (mine & 63)) & 1ull;
-            if (sent_mine) c2 += 1;
-        }
-        if (want < 0) {
-            if (got >= 0) c3 += 1;
-        } else if (got != want) {
-            c0 += 1;
-        } else if (a != root && (mine == want || ((once[(size_t)(want >> 6) * P + a] >> (want & 63)) & 1ull))) {
-            c1 += 1;                                       // it would never be passed on
-        } else {
-            value[(size_t)want * p + a] += value[(size_t)want * p + t];
-            c6 += 1;
-        }
-        if (mine >= 0) {
-            unsigned long long *set = sent_mine ? twice : once;
-            set[(size_t)(mine >> 6) * P + a] |= 1ull << (mine & 63);
-        }
-    }
-    add_stat(bstats, 0, c0);
-    add_stat(bstats, 1, c1);
-    add_stat(bstats, 2, c2);
-    add_stat(bstats, 3, c3);
-    add_stat(bstats, 6, c6);
+    RoundCounts c;
+    reduce_round(recv_k, send_k, value, once, twice, P, p, root, last, skip_k, shift, c);
+    add_round_counts(bstats, c);
     stats_end(bstats, stats);
+}
+
+// Rounds j1-1 down to j0 of the reduction in one cooperative launch (see broadcast_rounds_kernel).
+__global__ void __launch_bounds__(kFusedThreads, kFusedBlocks)
+reduce_rounds_kernel(const int8_t *__restrict__ recv_t, const int8_t *__restrict__ send_t,
+                     uint64_t *value, unsigned long long *once, unsigned long long *twice, size_t P,
+                     uint32_t p, uint32_t root, int last, const __grid_constant__ RoundPlan plan,
+                     long long j0, long long j1, GridBarrier *gb, unsigned long long barriers_before,
+                     unsigned long long *stats)
+{
+    __shared__ BlockStats64 bstats;
+    stats64_begin(bstats);
+    const long long i1 = plan.x + j1 - 1;
+    int k = (int)(i1 % plan.q);
+    int shift = (int)((i1 / plan.q) * plan.q - plan.x);
+    unsigned long long barriers = barriers_before;
+    bool failed = false;
+    RoundCounts c;                                         // 32 bits are enough: see broadcast_rounds_kernel
+    for (long long j = j1 - 1; j >= j0; --j) {
+        reduce_round(recv_t + (size_t)k * P, send_t + (size_t)k * P, value, once, twice, P, p, root, last,
+                     plan.skip[k], shift, c);
+        if (--k < 0) { k = plan.q - 1; shift -= plan.q; }
+        if (j > j0 && !grid_barrier(gb, ++barriers)) { failed = true; break; }
+    }
+    if (failed) return;
+    add_stat64(bstats, 0, c.c0);
+    add_stat64(bstats, 1, c.c1);
+    add_stat64(bstats, 2, c.c2);
+    add_stat64(bstats, 3, c.c3);
+    add_stat64(bstats, 6, c.c6);
+    stats64_end(bstats, stats);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -485,11 +699,63 @@ static int check_common(int32_t p, int32_t root, int64_t n, const void *recv, co
     return BCAST_OK;
 }
 
+// How the rounds of the single-root simulators are launched: one launch per round, or all rounds in
+// cooperative launches whose blocks meet between two rounds.  BCAST_SIMULATE_ROUNDS=launches|fused in
+// the environment, read once, or bcast_set_simulate_rounds; otherwise fused where the device allows it.
+static std::atomic<int> g_rounds_mode{-1};
+
+static int rounds_mode()
+{
+    int mode = g_rounds_mode.load(std::memory_order_relaxed);
+    if (mode >= 0) return mode;
+    mode = BCAST_ROUNDS_AUTO;
+    if (const char *env = getenv("BCAST_SIMULATE_ROUNDS")) {
+        if (strcmp(env, "launches") == 0) mode = BCAST_ROUNDS_LAUNCHES;
+        else if (strcmp(env, "fused") == 0) mode = BCAST_ROUNDS_FUSED;
+    }
+    int expected = -1;
+    g_rounds_mode.compare_exchange_strong(expected, mode, std::memory_order_relaxed);
+    return g_rounds_mode.load(std::memory_order_relaxed);
+}
+
+// Blocks of a cooperative launch of `kernel` that run all at once on the current device; 0 if the
+// device has no cooperative launches.
+static unsigned int cooperative_blocks(const void *kernel)
+{
+    int dev = 0, can = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&can, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !can)
+        return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kFusedThreads, 0) != cudaSuccess || per_sm <= 0)
+        return 0;
+    return (unsigned int)per_sm * (unsigned int)device_sm_count();
+}
+
+static RoundPlan round_plan(const Plan &plan)
+{
+    RoundPlan rp = {};
+    for (int k = 0; k < plan.q && k < 32; ++k) rp.skip[k] = plan.skip[k];
+    rp.q = plan.q;
+    rp.x = (int)plan.x;
+    return rp;
+}
+
+// Rounds of one cooperative launch: bounds the time a single kernel runs for huge n.
+constexpr int64_t kRoundsPerLaunch = 1 << 16;
+
 }  // namespace bcast_sim
 
 using namespace bcast_sim;
 
 extern "C" {
+
+int bcast_set_simulate_rounds(int mode)
+{
+    if (mode != BCAST_ROUNDS_AUTO && mode != BCAST_ROUNDS_LAUNCHES && mode != BCAST_ROUNDS_FUSED)
+        return BCAST_EINVAL_SHAPE;
+    g_rounds_mode.store(mode, std::memory_order_relaxed);
+    return BCAST_OK;
+}
 
 int64_t bcast_simulate_scratch_bytes(int32_t p, int64_t n, int reduction)
 {
@@ -521,46 +787,71 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
     unsigned long long *stats = reinterpret_cast<unsigned long long *>(stats_dev);
     if (cudaMemsetAsync(stats_dev, 0, 8 * sizeof(uint64_t), stream) != cudaSuccess) return BCAST_ECUDA;
     const unsigned int blocks = (unsigned int)(((int64_t)p + kThreads - 1) / kThreads);
-    // blocks of the arrival table go in slices of at most 65535 (the grid's y limit)
-    for (int64_t b0 = 0; b0 < n; b0 += 65535) {
-        const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
-        init_arrival_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(arrival_dev + (size_t)b0 * p, (uint32_t)p,
-                                                                       (uint32_t)root);
+    const GridBarrier *seal_stats_after = nullptr;
+    // -1 everywhere (all bytes 0xff), then 0 down the root's column
+    if (cudaMemsetAsync(arrival_dev, 0xff, (size_t)n * (size_t)p * sizeof(int32_t), stream) != cudaSuccess)
+        return BCAST_ECUDA;
+    root_arrival_kernel<<<(unsigned int)((n + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
+        arrival_dev, (uint32_t)p, (uint32_t)root, n);
+    if (q == 0) return cudaGetLastError() == cudaSuccess ? 0 : BCAST_ECUDA;
+    int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
+    int8_t *send_t = recv_t + (size_t)q * plan.P;
+    unsigned long long *held = reinterpret_cast<unsigned long long *>(send_t + (size_t)q * plan.P);
+    const int64_t rounds = n - 1 + q;
+    BroadcastFrame fr = {};
+    fr.arrival = arrival_dev;
+    fr.held = held;
+    fr.P = (size_t)plan.P;
+    fr.p = (uint32_t)p;
+    fr.root = (uint32_t)root;
+    fr.last = (int)(n - 1);
+    const unsigned int pblocks = (unsigned int)(plan.P / kThreads + (plan.P % kThreads != 0));
+    for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
+        const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
+        init_block_sets_kernel<<<dim3(pblocks, nw), kThreads, 0, stream>>>(
+            held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, (uint32_t)root, n - 64 * w0, 1);
     }
-    if (q > 0) {
-        int8_t *recv_t = reinterpret_cast<int8_t *>(scratch_dev) + kHeaderBytes;
-        int8_t *send_t = recv_t + (size_t)q * plan.P;
-        unsigned long long *held = reinterpret_cast<unsigned long long *>(send_t + (size_t)q * plan.P);
-        const unsigned int pblocks = (unsigned int)(plan.P / kThreads + (plan.P % kThreads != 0));
-        for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
-            const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
-            init_block_sets_kernel<<<dim3(pblocks, nw), kThreads, 0, stream>>>(
-                held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, (uint32_t)root, n - 64 * w0, 1);
+    transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
+        recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
+    const unsigned int resident = (unsigned int)device_sm_count() * 8u;
+    const int mode = rounds_mode();
+    const unsigned int together =
+        mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)broadcast_rounds_kernel);
+    if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
+    if (together != 0u) {
+        GridBarrier *gb = reinterpret_cast<GridBarrier *>(scratch_dev);
+        if (cudaMemsetAsync(gb, 0, sizeof(GridBarrier), stream) != cudaSuccess) return BCAST_ECUDA;
+        const unsigned int wanted = (unsigned int)(((int64_t)p + kFusedThreads - 1) / kFusedThreads);
+        const unsigned int grid = wanted < together ? wanted : together;
+        const int8_t *recv_c = recv_t, *send_c = send_t;
+        RoundPlan rp = round_plan(plan);
+        unsigned long long barriers = 0;
+        for (int64_t j0 = 0; j0 < rounds; j0 += kRoundsPerLaunch) {
+            long long first = j0, end = j0 + kRoundsPerLaunch < rounds ? j0 + kRoundsPerLaunch : rounds;
+            void *args[] = {&fr, &recv_c, &send_c, &rp, &first, &end, &gb, &barriers, &stats};
+            if (cudaLaunchCooperativeKernel((const void *)broadcast_rounds_kernel, dim3(grid), dim3(kFusedThreads),
+                                            args, 0, stream) != cudaSuccess)
+                return BCAST_ECUDA;
+            barriers += (unsigned long long)(end - first - 1);
         }
-        transpose_tables_kernel<<<dim3(blocks, 2), kThreads, 0, stream>>>(
-            recvblock_dev, sendblock_dev, recv_t, send_t, (uint32_t)p, q, (size_t)plan.P, stats);
-        const int64_t rounds = n - 1 + q;
-        const unsigned int resident = (unsigned int)device_sm_count() * 8u;
+        seal_stats_after = gb;
+    } else {
         const unsigned int round_blocks = blocks < resident ? blocks : resident;
         for (int64_t j = 0; j < rounds; ++j) {
             const int64_t i = plan.x + j;
             const int k = (int)(i % q);
-            const int64_t shift = (i / q) * q - plan.x;            // Theorem 1
+            const int64_t shift = (i / q) * q - plan.x;                // Theorem 1
             broadcast_round_kernel<<<round_blocks, kThreads, 0, stream>>>(
-                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, arrival_dev, held, (size_t)plan.P,
-                (uint32_t)p, (uint32_t)root, (int)(n - 1), plan.skip[k], (int)shift, (int32_t)(j + 1), stats);
+                fr, recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, plan.skip[k], (int)shift, (int32_t)(j + 1),
+                stats);
         }
     }
-    if (q > 0) {
-        const unsigned long long *held = reinterpret_cast<const unsigned long long *>(
-            reinterpret_cast<const int8_t *>(scratch_dev) + kHeaderBytes + 2 * (size_t)q * plan.P);
-        const unsigned int resident = (unsigned int)device_sm_count() * 8u;
-        for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
-            const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
-            count_missing_sets_kernel<<<dim3(blocks < resident ? blocks : resident, nw), kThreads, 0, stream>>>(
-                held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, n - 64 * w0, stats);
-        }
+    for (int64_t w0 = 0; w0 < set_words(n); w0 += 65535) {
+        const unsigned int nw = (unsigned int)(set_words(n) - w0 < 65535 ? set_words(n) - w0 : 65535);
+        count_missing_sets_kernel<<<dim3(blocks < resident ? blocks : resident, nw), kThreads, 0, stream>>>(
+            held + (size_t)w0 * plan.P, (size_t)plan.P, (uint32_t)p, n - 64 * w0, stats);
     }
+    if (seal_stats_after != nullptr) seal_stats_kernel<<<1, 32, 0, stream>>>(seal_stats_after, stats);
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
 }
@@ -597,20 +888,47 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
     const int64_t rounds = n - 1 + q;
     const unsigned int resident = (unsigned int)device_sm_count() * 8u;
     const unsigned int round_blocks = blocks < resident ? blocks : resident;
-    for (int64_t j = rounds - 1; j >= 0; --j) {                    // the broadcast's rounds, last one first
-        const int64_t i = plan.x + j;
-        const int k = (int)(i % q);
-        const int64_t shift = (i / q) * q - plan.x;
-        reduce_round_kernel<<<round_blocks, kThreads, 0, stream>>>(recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P,
-                                                             value_dev, once, twice, (size_t)plan.P, (uint32_t)p,
-                                                             (uint32_t)root, (int)(n - 1), plan.skip[k], (int)shift,
-                                                             stats);
+    const int mode = rounds_mode();
+    const unsigned int together =
+        mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)reduce_rounds_kernel);
+    if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
+    GridBarrier *gb = nullptr;
+    if (together != 0u) {
+        gb = reinterpret_cast<GridBarrier *>(scratch_dev);
+        if (cudaMemsetAsync(gb, 0, sizeof(GridBarrier), stream) != cudaSuccess) return BCAST_ECUDA;
+        const unsigned int wanted = (unsigned int)(((int64_t)p + kFusedThreads - 1) / kFusedThreads);
+        const unsigned int grid = wanted < together ? wanted : together;
+        const int8_t *recv_c = recv_t, *send_c = send_t;
+        size_t P = (size_t)plan.P;
+        uint32_t up = (uint32_t)p, uroot = (uint32_t)root;
+        int last = (int)(n - 1);
+        RoundPlan rp = round_plan(plan);
+        unsigned long long barriers = 0;
+        for (int64_t j1 = rounds; j1 > 0; j1 -= kRoundsPerLaunch) {    // the broadcast's rounds, last one first
+            long long end = j1, first = j1 > kRoundsPerLaunch ? j1 - kRoundsPerLaunch : 0;
+            void *args[] = {&recv_c, &send_c, &value_dev, &once, &twice, &P, &up, &uroot, &last, &rp, &first, &end,
+                            &gb, &barriers, &stats};
+            if (cudaLaunchCooperativeKernel((const void *)reduce_rounds_kernel, dim3(grid), dim3(kFusedThreads), args, 0,
+                                            stream) != cudaSuccess)
+                return BCAST_ECUDA;
+            barriers += (unsigned long long)(end - first - 1);
+        }
+    } else {
+        for (int64_t j = rounds - 1; j >= 0; --j) {                // the broadcast's rounds, last one first
+            const int64_t i = plan.x + j;
+            const int k = (int)(i % q);
+            const int64_t shift = (i / q) * q - plan.x;
+            reduce_round_kernel<<<round_blocks, kThreads, 0, stream>>>(
+                recv_t + (size_t)k * plan.P, send_t + (size_t)k * plan.P, value_dev, once, twice, (size_t)plan.P,
+                (uint32_t)p, (uint32_t)root, (int)(n - 1), plan.skip[k], (int)shift, stats);
+        }
     }
     for (int64_t b0 = 0; b0 < n; b0 += 65535) {
         const unsigned int nb = (unsigned int)(n - b0 < 65535 ? n - b0 : 65535);
         reduce_finish_kernel<<<dim3(blocks, nb), kThreads, 0, stream>>>(
             value_dev, once, twice, (size_t)plan.P, result_dev, (uint32_t)p, (uint32_t)root, b0, stats);
     }
+    if (gb != nullptr) seal_stats_kernel<<<1, 32, 0, stream>>>(gb, stats);
     if (cudaGetLastError() != cudaSuccess) return BCAST_ECUDA;
     return q;
 }

@@ -20,6 +20,14 @@ def _need_gpu():
         pytest.skip("no CUDA device")
 
 
+@pytest.fixture(params=["launches", "fused"])
+def rounds(request):
+    """The single-root simulators with one launch per round, and with all rounds in cooperative launches."""
+    bs.bcast_set_simulate_rounds({"launches": bs.BCAST_ROUNDS_LAUNCHES, "fused": bs.BCAST_ROUNDS_FUSED}[request.param])
+    yield request.param
+    bs.bcast_set_simulate_rounds(bs.BCAST_ROUNDS_AUTO)
+
+
 def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
@@ -40,7 +48,7 @@ def check_broadcast(p, root, n, recv, send):
 
 # ------------------------------------------------------------------ broadcast
 @pytest.mark.parametrize("p", [1, 2, 3, 17, 255, 256, 257, 1000, 4099])
-def test_broadcast_small_p_every_phase_offset(p):
+def test_broadcast_small_p_every_phase_offset(p, rounds):
     q = oracle.q_of(p)
     for root in sorted({0, p // 3, p - 1}):
         recv, send = oracle.schedule_table(p, root)
@@ -50,7 +58,7 @@ def test_broadcast_small_p_every_phase_offset(p):
             assert stats[7] == (n - 1 + q if p > 1 else 0)
 
 
-def test_broadcast_config1_on_gpu_tables():
+def test_broadcast_config1_on_gpu_tables(rounds):
     # config 1: p = 1000, 8 blocks over 17 rounds, on the tables the GPU itself computed
     p, n = workloads.P_SMALL, 8
     recv, send = bs.schedule(p, 0)
@@ -61,7 +69,7 @@ def test_broadcast_config1_on_gpu_tables():
     assert np.array_equal(arrival.cpu().numpy(), want_arrival)
 
 
-def test_broadcast_medium_p_many_blocks():
+def test_broadcast_medium_p_many_blocks(rounds):
     # several tiles of 256 processors with a ragged tail, more blocks than one phase, other root
     p, root, n = 70001, 12345, 40
     recv, send = oracle.schedule_table(p, root)
@@ -69,7 +77,7 @@ def test_broadcast_medium_p_many_blocks():
     assert stats[:6].tolist() == [0] * 6
 
 
-def test_broadcast_config2_on_gpu_tables_properties():
+def test_broadcast_config2_on_gpu_tables_properties(rounds):
     # config 2's p on the GPU's own tables: too large for the oracle's simulation in seconds, so the
     # facts that hold at any size are checked, and sampled processors against Theorem 1 row by row
     p, n = workloads.P_MEDIUM, 24
@@ -104,7 +112,7 @@ def damaged_tables(p, root, seed, count):
 
 
 @pytest.mark.parametrize("p,root,n,count", [(37, 4, 9, 1), (300, 0, 5, 6), (1000, 77, 13, 40), (5000, 1, 3, 500)])
-def test_broadcast_damaged_tables_same_findings(p, root, n, count):
+def test_broadcast_damaged_tables_same_findings(p, root, n, count, rounds):
     recv, send = damaged_tables(p, root, p + n, count)
     stats = check_broadcast(p, root, n, recv, send)
     assert sum(int(v) for v in stats[:6]) > 0
@@ -158,7 +166,7 @@ def check_reduce(p, root, n, recv, send, value):
 
 
 @pytest.mark.parametrize("p", [1, 2, 3, 17, 256, 257, 1000, 4099])
-def test_reduce_small_p(p):
+def test_reduce_small_p(p, rounds):
     q = oracle.q_of(p)
     for root in sorted({0, p // 3, p - 1}):
         recv, send = oracle.schedule_table(p, root)
@@ -170,7 +178,7 @@ def test_reduce_small_p(p):
             assert stats[:6].tolist() == [0] * 6 and stats[6] == (p - 1) * n
 
 
-def test_reduce_medium_p_on_gpu_tables():
+def test_reduce_medium_p_on_gpu_tables(rounds):
     p, root, n = 70001, 4321, 30
     recv, send = bs.schedule(p, root)
     value = contributions(p, n, 11)
@@ -184,7 +192,7 @@ def test_reduce_medium_p_on_gpu_tables():
 
 
 @pytest.mark.parametrize("p,root,n,count", [(37, 4, 9, 1), (300, 0, 5, 6), (1000, 77, 13, 40)])
-def test_reduce_damaged_tables_same_findings(p, root, n, count):
+def test_reduce_damaged_tables_same_findings(p, root, n, count, rounds):
     recv, send = damaged_tables(p, root, 3 * p + n, count)
     value = contributions(p, n, 5)
     _, stats = check_reduce(p, root, n, recv, send, value)
@@ -225,7 +233,7 @@ def test_shifted_tables_ranges_and_unaligned():
     assert e.value.code == -6
 
 
-def test_more_blocks_than_one_launch_grid_holds():
+def test_more_blocks_than_one_launch_grid_holds(rounds):
     # n above 65535: the per-block launches (arrival set-up, the reduction's last pass) go in slices
     p, root, n = 5, 3, 70001
     recv, send = oracle.schedule_table(p, root)
@@ -236,6 +244,18 @@ def test_more_blocks_than_one_launch_grid_holds():
     with np.errstate(over="ignore"):
         assert result.tolist() == value.sum(axis=1, dtype=np.uint64).tolist()
     assert rstats[:6].tolist() == [0] * 6
+
+
+def test_more_rounds_than_one_cooperative_launch_holds_on_several_blocks(rounds):
+    # n - 1 + q above 65536 rounds on four blocks of processors: the fused form goes in two launches, and
+    # the blocks' meeting counter carries over from the first to the second
+    p, root, n = 1000, 7, 65600
+    recv, send = oracle.schedule_table(p, root)
+    stats = check_broadcast(p, root, n, recv, send)
+    assert stats[:6].tolist() == [0] * 6 and stats[6] == (p - 1) * n and stats[7] == n - 1 + 10
+    value = contributions(p, n, 2)
+    result, rstats = check_reduce(p, root, n, recv, send, value)
+    assert rstats[:6].tolist() == [0] * 6 and rstats[6] == (p - 1) * n
 
 
 # ------------------------------------------------------------------ all roots at once: Algorithm 7 and its reversal
