@@ -213,7 +213,7 @@ def workload_label(mode: str, p: int, q: int, blocks: int = 0) -> str:
 def oracle_other_modes(p: int):
     """The oracle's other routes, timed beside the window mode (single thread, as it stands):
     receive rows alone on a window of the same p, and the all-ranks route (receive rows by Algorithm 5 for
-    every rank, send rows gathered from them: one search per rank) on BASELINE config 2 in full."""
+    every rank, send rows gathered from them: one search per rank) on configuration 2 (p = 2^20 + 1) in full."""
     import oracle
     from paper_2407_18004_b200 import workloads
     rows = min(p, 2 ** 21)
@@ -464,7 +464,7 @@ def measure_store_ceiling(bs, torch, recv, send, stream):
 
 
 def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
-    """The other BASELINE configurations and the library's other table forms, measured in the same run (same
+    """The other benchmark configurations and the library's other table forms, measured in the same run (same
     device buffers, same clock sampling window is not repeated: short runs).  Each entry: mean ms per launch, the
     workload's own throughput, and the roofline fraction with its bound."""
     from paper_2407_18004_b200 import workloads
@@ -491,7 +491,7 @@ def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
 
     table_entry("config2_p=2^20+1", workloads.P_MEDIUM,
                 lambda p, q, r, s_: bs.bcast_schedule(p, 0, 0, p, r, s_, stream), 5, 60,
-                "all ranks of p=%d (q=%d), root 0 (BASELINE config 2); tables larger than L2, launches back to back")
+                "all ranks of p=%d (q=%d), root 0 (configuration 2); tables larger than L2, launches back to back")
     table_entry("ordinary_p=123456789", 123456789,
                 lambda p, q, r, s_: bs.bcast_schedule(p, 0, 0, p, r, s_, stream), 10, 1,
                 "all ranks of p=%d (q=%d), root 0: a p with no special form")
@@ -521,7 +521,7 @@ def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
     ach = insts / (mean_ms * 1e-3) / 1e9 if insts else None
     out["config5_batch_2^24"] = {
         "workload": "2^24 queries, p log-uniform in [2, 2^31-1], rank and root uniform, seed 0, rows padded to 31 "
-                    "(BASELINE config 5)", "ms": mean_ms, "ms_min": min_ms, "value": nq / (mean_ms * 1e-3),
+                    "(configuration 5)", "ms": mean_ms, "ms_min": min_ms, "value": nq / (mean_ms * 1e-3),
         "unit": "queries/s", "bytes_per_launch": nq * (2 * 31 * 4 + 12),
         "hbm_write_gbs": nq * 2 * 31 * 4 / (mean_ms * 1e-3) / 1e9,
         "roofline": {"bound": "alu", "achieved": ach, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
@@ -543,7 +543,7 @@ def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
     ach = insts / (mean_ms * 1e-3) / 1e9 if insts else None
     out["config4_sweep_2_65536"] = {
         "workload": "every p in [2, 65536], all ranks, root 0: tables built and checked on the device, one checksum "
-                    "per p (BASELINE config 4)", "ms": mean_ms, "ms_min": min_ms, "value": units / (mean_ms * 1e-3),
+                    "per p (configuration 4)", "ms": mean_ms, "ms_min": min_ms, "value": units / (mean_ms * 1e-3),
         "unit": "rank-schedules/s", "fail_counts": fails.tolist(),
         "roofline": {"bound": "alu", "achieved": ach, "peak": ISSUE_PEAK_GINST, "unit": "G warp-inst/s",
                      "frac": ach / ISSUE_PEAK_GINST if ach else None, "warp_instructions_per_launch": insts}}
@@ -924,7 +924,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
-                    help="skip the other BASELINE configurations that the default run measures beside the headline")
+                    help="skip the other benchmark configurations that the default run measures beside the headline")
     args = ap.parse_args()
     if args.mode in OTHER_MODES:
         if args.workload == "p=2^27-1":
