@@ -281,7 +281,7 @@ int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev
  * Limits: n < 2^31 - 64; n * p int32 cells must fit the caller's memory.
  *
  * The n-1+q rounds run either as one small launch each or, by default where the
- * device has cooperative launches, inside cooperative launches of up to 65536
+ * device has cooperative launches (and grants this one), inside cooperative launches of up to 65536
  * rounds whose blocks meet at a counter in the scratch between two rounds (a
  * round of 2^20 processors is too short to pay for a launch of its own).  That
  * wait is bounded: should a block see no progress for about two seconds (all

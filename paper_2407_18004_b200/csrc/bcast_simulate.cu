@@ -818,7 +818,8 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
     const unsigned int together =
         mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)broadcast_rounds_kernel);
     if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
-    if (together != 0u) {
+    bool fused = together != 0u;
+    if (fused) {
         GridBarrier *gb = reinterpret_cast<GridBarrier *>(scratch_dev);
         if (cudaMemsetAsync(gb, 0, sizeof(GridBarrier), stream) != cudaSuccess) return BCAST_ECUDA;
         const unsigned int wanted = (unsigned int)(((int64_t)p + kFusedThreads - 1) / kFusedThreads);
@@ -830,12 +831,19 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
             long long first = j0, end = j0 + kRoundsPerLaunch < rounds ? j0 + kRoundsPerLaunch : rounds;
             void *args[] = {&fr, &recv_c, &send_c, &rp, &first, &end, &gb, &barriers, &stats};
             if (cudaLaunchCooperativeKernel((const void *)broadcast_rounds_kernel, dim3(grid), dim3(kFusedThreads),
-                                            args, 0, stream) != cudaSuccess)
-                return BCAST_ECUDA;
+                                            args, 0, stream) != cudaSuccess) {
+                // refused before anything ran (the device is shared, say): one launch per round instead,
+                // unless the fused form was asked for
+                if (j0 != 0 || mode == BCAST_ROUNDS_FUSED) return BCAST_ECUDA;
+                (void)cudaGetLastError();
+                fused = false;
+                break;
+            }
             barriers += (unsigned long long)(end - first - 1);
         }
-        seal_stats_after = gb;
-    } else {
+        if (fused) seal_stats_after = gb;
+    }
+    if (!fused) {
         const unsigned int round_blocks = blocks < resident ? blocks : resident;
         for (int64_t j = 0; j < rounds; ++j) {
             const int64_t i = plan.x + j;
@@ -893,7 +901,8 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
         mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)reduce_rounds_kernel);
     if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
     GridBarrier *gb = nullptr;
-    if (together != 0u) {
+    bool fused = together != 0u;
+    if (fused) {
         gb = reinterpret_cast<GridBarrier *>(scratch_dev);
         if (cudaMemsetAsync(gb, 0, sizeof(GridBarrier), stream) != cudaSuccess) return BCAST_ECUDA;
         const unsigned int wanted = (unsigned int)(((int64_t)p + kFusedThreads - 1) / kFusedThreads);
@@ -909,11 +918,17 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
             void *args[] = {&recv_c, &send_c, &value_dev, &once, &twice, &P, &up, &uroot, &last, &rp, &first, &end,
                             &gb, &barriers, &stats};
             if (cudaLaunchCooperativeKernel((const void *)reduce_rounds_kernel, dim3(grid), dim3(kFusedThreads), args, 0,
-                                            stream) != cudaSuccess)
-                return BCAST_ECUDA;
+                                            stream) != cudaSuccess) {
+                if (j1 != rounds || mode == BCAST_ROUNDS_FUSED) return BCAST_ECUDA;
+                (void)cudaGetLastError();                          // refused before anything ran: see the broadcast
+                fused = false;
+                gb = nullptr;
+                break;
+            }
             barriers += (unsigned long long)(end - first - 1);
         }
-    } else {
+    }
+    if (!fused) {
         for (int64_t j = rounds - 1; j >= 0; --j) {                // the broadcast's rounds, last one first
             const int64_t i = plan.x + j;
             const int k = (int)(i % q);
