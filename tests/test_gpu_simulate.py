@@ -77,10 +77,12 @@ def test_broadcast_medium_p_many_blocks(rounds):
     assert stats[:6].tolist() == [0] * 6
 
 
-def test_broadcast_config2_on_gpu_tables_properties(rounds):
-    # config 2's p on the GPU's own tables: too large for the oracle's simulation in seconds, so the
-    # facts that hold at any size are checked, and sampled processors against Theorem 1 row by row
-    p, n = workloads.P_MEDIUM, 24
+@pytest.mark.parametrize("n", [24, 64])
+def test_broadcast_config2_on_gpu_tables_properties(rounds, n):
+    # config 2's p on the GPU's own tables (n = 64 is the benchmark's simulation): too large for the oracle's
+    # simulation in seconds, so the facts that hold at any size are checked, and sampled processors against
+    # Theorem 1 row by row
+    p = workloads.P_MEDIUM
     q = bs.bcast_q(p)
     recv, send = bs.schedule(p, 0)
     arrival, stats = bs.simulate_broadcast(p, 0, n, recv, send)
@@ -189,6 +191,20 @@ def test_reduce_medium_p_on_gpu_tables(rounds):
     assert u64(stats).tolist() == [0, 0, 0, 0, 0, 0, (p - 1) * n, 0]
     orecv, osend = oracle.schedule_table(p, root)
     check_reduce(p, root, n, orecv, osend, value)
+
+
+def test_reduce_config2_on_gpu_tables_sums(rounds):
+    # the benchmark's reduction (config 2's p, 64 blocks) on the GPU's own tables: the root must end up with the
+    # wrapping sum of every block's contributions, every partial result combined exactly once
+    p, n = workloads.P_MEDIUM, 64
+    recv, send = bs.schedule(p, 0)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    value = torch.randint(0, 2 ** 62, (n, p), dtype=torch.int64, device="cuda", generator=gen)
+    result, stats = bs.simulate_reduce(p, 0, n, recv, send, value)
+    torch.cuda.synchronize()
+    assert torch.equal(result, value.sum(dim=1))               # int64 sums wrap like the uint64 ones
+    assert u64(stats).tolist() == [0, 0, 0, 0, 0, 0, (p - 1) * n, 0]
 
 
 @pytest.mark.parametrize("p,root,n,count", [(37, 4, 9, 1), (300, 0, 5, 6), (1000, 77, 13, 40)])
