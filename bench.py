@@ -506,6 +506,42 @@ def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
                 lambda p, q, r, s_: bs.bcast_schedule_shifted(p, 0, 64, 0, p, r, s_, stream), 10, 1,
                 "all ranks of p=%d (q=%d), root 0, rows after Algorithm 1's preamble for n=64 blocks")
 
+    # the tables in use: Algorithm 1 and its reversal by all processors of configuration 2's p, 64 blocks, on
+    # tables left by a launch in the same buffers; state and scratch come out of the send buffer's tail
+    p, n = workloads.P_MEDIUM, 64
+    q, r, s_ = tables(p)
+    bs.bcast_schedule(p, 0, 0, p, r, s_, stream)
+    rounds = n - 1 + q
+    spare = flat_s[(p * q + 3) // 4 * 4:]                  # from a 16-byte boundary on
+    arrival = spare[:n * p].view(n, p)
+    need = bs.bcast_simulate_scratch_bytes(p, n, True)
+    n_words = 2 * n * p + n + 8 + (need + 7) // 8
+    words = spare[n * p:n * p + 2 * n_words].view(torch.int64)     # n * p is a multiple of 4: still on a 16-byte boundary
+    value, contrib = words[:n * p].view(n, p), words[n * p:2 * n * p].view(n, p)
+    result, stats = words[2 * n * p:2 * n * p + n], words[2 * n * p + n:2 * n * p + n + 8]
+    scratch = words[2 * n * p + n + 8:].view(torch.uint8)[:need]           # an even number of words in: 16-byte aligned
+    contrib.random_(0, 2 ** 62)
+
+    def reduce_step():
+        value.copy_(contrib)
+        bs.bcast_simulate_reduce(p, 0, n, r, s_, value, result, stats, scratch, stream)
+
+    for name, fn, nbytes, what in (
+            ("simulate_n=64_p=2^20+1", lambda: bs.bcast_simulate_broadcast(p, 0, n, r, s_, arrival, stats, scratch, stream),
+             p * (10 * q + 8 * n + rounds * 14), "Algorithm 1 by all processors of p=%d (q=%d), 64 blocks, %d rounds"),
+            ("reduce_n=64_p=2^20+1", reduce_step, p * (10 * q + 18 * n + rounds * 30),
+             "Observation 1.3's reduction by all processors of p=%d (q=%d), 64 blocks, %d rounds, contributions copied in")):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        mean_ms, min_ms = time_launches(torch, stream, fn, 10)
+        gbs = nbytes / (mean_ms * 1e-3) / 1e9
+        out[name] = {"workload": what % (p, q, rounds), "ms": mean_ms, "ms_min": min_ms,
+                     "value": (p - 1) * n / (mean_ms * 1e-3), "unit": "blocks/s", "bytes_per_step": nbytes,
+                     "stats": stats.tolist(),
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                  "note": "algorithmic bytes of the whole step (all of its launches) over its time"}}
+
     # config 5: 2^24 independent queries (rows padded to 31), outputs in the same buffers
     nq = 2 ** 24
     hp, hr, ho = workloads.query_batch(nq, seed=0)
