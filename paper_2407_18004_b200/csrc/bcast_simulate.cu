@@ -11,14 +11,18 @@
 //     processor from each table, consecutive processors from consecutive addresses, and the
 //     2q*P bytes stay in L2 over the n-1+q rounds.  Entries outside [-q, q-1] are counted
 //     and stored as kInvalid, which moves nothing in any round.
-//   * One thread per processor, one launch per round, all on the caller's stream.  Nothing
-//     waits on another block inside a launch.
-//   * Broadcast state is arrival[b][a], the round in which processor a got block b.  A
-//     sender "held the block before the round" iff its arrival is in [0, round); a value
-//     written during the round is >= round, so concurrent readers decide the same way
-//     whether or not they see it: one buffer, no race in the outcome.
-//   * Reduction state is value[b][a] plus a saturating count sent[b][a]; a receiver reads its
-//     to-processor's partial result in place (see reduce_round_kernel for why the outcome
+//   * One thread per processor on a grid that strides over the processors, all on the
+//     caller's stream.  The single-root simulators run their rounds inside cooperative
+//     launches whose blocks meet between two rounds (a bounded wait; see grid_barrier), or
+//     as one launch per round; the all-roots ones as one launch per round, in which nothing
+//     waits on another block.
+//   * Broadcast state is arrival[b][a], the round in which processor a got block b, and a bit
+//     per (processor, block), held[w][a], which is what a round reads.  A sender "held the
+//     block before the round" iff its bit was set before; where the bit may be changing in
+//     this very round the arrival cell decides: a value written during the round is >= round,
+//     so concurrent readers decide the same way whether or not they see it.
+//   * Reduction state is value[b][a] plus two bit sets (sent once, sent twice); a receiver reads
+//     its to-processor's partial result in place (see reduce_round for why the outcome
 //     does not depend on the order of the threads).
 //   * Counters are summed per warp with redux, per block in shared memory, and added to the
 //     64-bit statistics with one atomic per block and counter that is not zero.
