@@ -279,7 +279,7 @@ struct GridBarrier {
 };
 static_assert(sizeof(GridBarrier) <= kHeaderBytes, "the barrier lives in the scratch header");
 
-constexpr unsigned int kBarrierSpins = 1u << 23;
+constexpr unsigned int kBarrierSpins = 1u << 21;      // a poll and its pause take about a microsecond
 #ifndef BCAST_FUSED_THREADS
 #define BCAST_FUSED_THREADS 1024
 #endif
