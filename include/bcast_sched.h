@@ -73,6 +73,10 @@ extern "C" {
 #define BCAST_ROUNDS_AUTO      0        /* fused where the device has cooperative launches (default) */
 #define BCAST_ROUNDS_LAUNCHES  1        /* one kernel launch per communication round                  */
 #define BCAST_ROUNDS_FUSED     2        /* all rounds in cooperative launches, blocks meet per round   */
+#define BCAST_ROUNDS_FUSED_MISS 3       /* for tests of the bounded wait: BCAST_ROUNDS_FUSED whose blocks */
+                                        /* wait for one block more than there are; every call with more   */
+                                        /* than one round ends, after a second or two, with all eight   */
+                                        /* statistics words UINT64_MAX                                     */
 
 #define BCAST_STATIC_SWEEP_BYTES  (8u << 20)   /* built-in scratch of bcast_verify_sweep_static */
 #define BCAST_STATIC_SWEEP_MAX_P  65536        /* largest p_hi it accepts                       */
@@ -284,7 +288,7 @@ int bcast_verify_sweep_static(int32_t p_lo, int32_t p_hi, uint64_t *checksum_dev
  * device has cooperative launches (and grants this one), inside cooperative launches of up to 65536
  * rounds whose blocks meet at a counter in the scratch between two rounds (a
  * round of 2^20 processors is too short to pay for a launch of its own).  That
- * wait is bounded: should a block see no progress for about two seconds (all
+ * wait is bounded: should a block see no progress for a second or two (all
  * blocks of a cooperative launch are resident, so this is not expected), every
  * block stops and ALL EIGHT statistics words are set to UINT64_MAX; arrival_dev
  * is then unspecified.  Both forms give the same arrival table and statistics.

@@ -20,7 +20,7 @@ BCAST_MAX_Q = 31
 BCAST_STATIC_SWEEP_MAX_P = 65536
 BCAST_UNRESOLVED = -128
 BCAST_SHAPE_AUTO, BCAST_SHAPE_BLOCK, BCAST_SHAPE_WARPS, BCAST_SHAPE_LOWFRAME, BCAST_SHAPE_WARPS_TIGHT = -1, 0, 1, 2, 3
-BCAST_ROUNDS_AUTO, BCAST_ROUNDS_LAUNCHES, BCAST_ROUNDS_FUSED = 0, 1, 2
+BCAST_ROUNDS_AUTO, BCAST_ROUNDS_LAUNCHES, BCAST_ROUNDS_FUSED, BCAST_ROUNDS_FUSED_MISS = 0, 1, 2, 3
 
 _lib = None
 

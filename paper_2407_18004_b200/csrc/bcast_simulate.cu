@@ -271,7 +271,7 @@ broadcast_round_kernel(const __grid_constant__ BroadcastFrame fr, const int8_t *
 // The blocks of a cooperative launch (all resident at once, or the launch is refused) meet between
 // two rounds at a counter in the caller's scratch: every block adds one after its threads' writes
 // are fenced, and waits until all blocks of the round have.  The wait is bounded: a block that
-// sees nothing for about two seconds raises `failed`, every block leaves its loop, and the
+// sees nothing for a second or two raises `failed`, every block leaves its loop, and the
 // statistics are overwritten with all-ones by seal_stats_kernel.
 struct GridBarrier {
     unsigned long long arrived;            // blocks that have reached a barrier, over all barriers of the call
@@ -292,12 +292,12 @@ constexpr int kFusedBlocks = BCAST_FUSED_BLOCKS;       // resident per SM
 // `index` = this barrier's number in the call, from 1.  The arrival is a release (the block's
 // writes, ordered before it by the block barrier, are visible to whoever sees the count) and, for
 // the last block in, an acquire; the others' wait is an acquire.
-__device__ __forceinline__ bool grid_barrier(GridBarrier *gb, unsigned long long index)
+__device__ __forceinline__ bool grid_barrier(GridBarrier *gb, unsigned long long index, unsigned int blocks)
 {
     __shared__ int through;
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned long long target = index * gridDim.x;
+        const unsigned long long target = index * blocks;
         unsigned long long seen;
         asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], 1;" : "=l"(seen) : "l"(&gb->arrived) : "memory");
         bool good = seen + 1ull >= target;
@@ -323,6 +323,7 @@ struct RoundPlan {
     uint32_t skip[32];
     int q;
     int x;
+    unsigned int blocks;                   // blocks a barrier waits for: the grid's (one more in the test of the wait's limit)
 };
 
 // Counters of a block over many rounds (64 bits: 2^31 rounds of a few thousand processors).
@@ -373,7 +374,7 @@ broadcast_rounds_kernel(const __grid_constant__ BroadcastFrame fr, const int8_t 
         broadcast_round(fr, recv_t + (size_t)k * fr.P, send_t + (size_t)k * fr.P, plan.skip[k], shift, (int32_t)(j + 1), c);
         if (c.c6 != delivered_before) last_delivery = (unsigned int)(j + 1);
         if (++k == plan.q) { k = 0; shift += plan.q; }
-        if (j + 1 < j1 && !grid_barrier(gb, ++barriers)) { failed = true; break; }
+        if (j + 1 < j1 && !grid_barrier(gb, ++barriers, plan.blocks)) { failed = true; break; }
     }
     if (failed) return;
     add_stat64(bstats, 0, c.c0);
@@ -503,7 +504,7 @@ reduce_rounds_kernel(const int8_t *__restrict__ recv_t, const int8_t *__restrict
         reduce_round(recv_t + (size_t)k * P, send_t + (size_t)k * P, value, once, twice, P, p, root, last,
                      plan.skip[k], shift, c);
         if (--k < 0) { k = plan.q - 1; shift -= plan.q; }
-        if (j > j0 && !grid_barrier(gb, ++barriers)) { failed = true; break; }
+        if (j > j0 && !grid_barrier(gb, ++barriers, plan.blocks)) { failed = true; break; }
     }
     if (failed) return;
     add_stat64(bstats, 0, c.c0);
@@ -755,7 +756,8 @@ extern "C" {
 
 int bcast_set_simulate_rounds(int mode)
 {
-    if (mode != BCAST_ROUNDS_AUTO && mode != BCAST_ROUNDS_LAUNCHES && mode != BCAST_ROUNDS_FUSED)
+    if (mode != BCAST_ROUNDS_AUTO && mode != BCAST_ROUNDS_LAUNCHES && mode != BCAST_ROUNDS_FUSED &&
+        mode != BCAST_ROUNDS_FUSED_MISS)
         return BCAST_EINVAL_SHAPE;
     g_rounds_mode.store(mode, std::memory_order_relaxed);
     return BCAST_OK;
@@ -821,7 +823,7 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
     const int mode = rounds_mode();
     const unsigned int together =
         mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)broadcast_rounds_kernel);
-    if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
+    if ((mode == BCAST_ROUNDS_FUSED || mode == BCAST_ROUNDS_FUSED_MISS) && together == 0u) return BCAST_ECUDA;
     bool fused = together != 0u;
     if (fused) {
         GridBarrier *gb = reinterpret_cast<GridBarrier *>(scratch_dev);
@@ -830,6 +832,7 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
         const unsigned int grid = wanted < together ? wanted : together;
         const int8_t *recv_c = recv_t, *send_c = send_t;
         RoundPlan rp = round_plan(plan);
+        rp.blocks = grid + (mode == BCAST_ROUNDS_FUSED_MISS ? 1u : 0u);
         unsigned long long barriers = 0;
         for (int64_t j0 = 0; j0 < rounds; j0 += kRoundsPerLaunch) {
             long long first = j0, end = j0 + kRoundsPerLaunch < rounds ? j0 + kRoundsPerLaunch : rounds;
@@ -838,7 +841,7 @@ int bcast_simulate_broadcast(int32_t p, int32_t root, int64_t n,
                                             args, 0, stream) != cudaSuccess) {
                 // refused before anything ran (the device is shared, say): one launch per round instead,
                 // unless the fused form was asked for
-                if (j0 != 0 || mode == BCAST_ROUNDS_FUSED) return BCAST_ECUDA;
+                if (j0 != 0 || mode != BCAST_ROUNDS_AUTO) return BCAST_ECUDA;
                 (void)cudaGetLastError();
                 fused = false;
                 break;
@@ -903,7 +906,7 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
     const int mode = rounds_mode();
     const unsigned int together =
         mode == BCAST_ROUNDS_LAUNCHES ? 0u : cooperative_blocks((const void *)reduce_rounds_kernel);
-    if (mode == BCAST_ROUNDS_FUSED && together == 0u) return BCAST_ECUDA;
+    if ((mode == BCAST_ROUNDS_FUSED || mode == BCAST_ROUNDS_FUSED_MISS) && together == 0u) return BCAST_ECUDA;
     GridBarrier *gb = nullptr;
     bool fused = together != 0u;
     if (fused) {
@@ -916,6 +919,7 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
         uint32_t up = (uint32_t)p, uroot = (uint32_t)root;
         int last = (int)(n - 1);
         RoundPlan rp = round_plan(plan);
+        rp.blocks = grid + (mode == BCAST_ROUNDS_FUSED_MISS ? 1u : 0u);
         unsigned long long barriers = 0;
         for (int64_t j1 = rounds; j1 > 0; j1 -= kRoundsPerLaunch) {    // the broadcast's rounds, last one first
             long long end = j1, first = j1 > kRoundsPerLaunch ? j1 - kRoundsPerLaunch : 0;
@@ -923,7 +927,7 @@ int bcast_simulate_reduce(int32_t p, int32_t root, int64_t n,
                             &gb, &barriers, &stats};
             if (cudaLaunchCooperativeKernel((const void *)reduce_rounds_kernel, dim3(grid), dim3(kFusedThreads), args, 0,
                                             stream) != cudaSuccess) {
-                if (j1 != rounds || mode == BCAST_ROUNDS_FUSED) return BCAST_ECUDA;
+                if (j1 != rounds || mode != BCAST_ROUNDS_AUTO) return BCAST_ECUDA;
                 (void)cudaGetLastError();                          // refused before anything ran: see the broadcast
                 fused = false;
                 gb = nullptr;

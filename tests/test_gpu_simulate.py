@@ -274,6 +274,27 @@ def test_more_rounds_than_one_cooperative_launch_holds_on_several_blocks(rounds)
     assert rstats[:6].tolist() == [0] * 6 and rstats[6] == (p - 1) * n
 
 
+def test_bounded_wait_runs_out_and_says_so():
+    # the blocks of the fused form are told to wait for one block more than there are: every wait gives up after
+    # about two seconds, every block stops, all eight statistics words come back as all-ones, and the context
+    # is as usable as before
+    p, n = 3000, 4                                         # three blocks of 1024 threads, 15 rounds
+    recv, send = bs.schedule(p, 0)
+    value = dev(contributions(p, n, 3).view(np.int64))
+    bs.bcast_set_simulate_rounds(bs.BCAST_ROUNDS_FUSED_MISS)
+    try:
+        _, stats = bs.simulate_broadcast(p, 0, n, recv, send)
+        _, rstats = bs.simulate_reduce(p, 0, n, recv, send, value)
+        torch.cuda.synchronize()
+    finally:
+        bs.bcast_set_simulate_rounds(bs.BCAST_ROUNDS_AUTO)
+    assert u64(stats).tolist() == [2 ** 64 - 1] * 8
+    assert u64(rstats).tolist() == [2 ** 64 - 1] * 8
+    orecv, osend = oracle.schedule_table(p, 0)
+    stats = check_broadcast(p, 0, n, orecv, osend)
+    assert stats[:6].tolist() == [0] * 6 and stats[6] == (p - 1) * n
+
+
 # ------------------------------------------------------------------ all roots at once: Algorithm 7 and its reversal
 def check_all(p, n, recv0, send0, tables_from_algorithm7):
     """The device gets the root-0 tables; the oracle takes every processor's tables from Algorithm 7's own

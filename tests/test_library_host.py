@@ -96,7 +96,7 @@ def test_host_argument_errors():
         bs.bcast_round_block(4, 3, -1, [0, 0, 0, 0])
     assert e.value.code == -7
     with pytest.raises(bs.BcastError) as e:
-        bs.bcast_set_simulate_rounds(3)
+        bs.bcast_set_simulate_rounds(4)
     assert e.value.code == -12
     for mode in (bs.BCAST_ROUNDS_FUSED, bs.BCAST_ROUNDS_LAUNCHES, bs.BCAST_ROUNDS_AUTO):
         assert bs.bcast_set_simulate_rounds(mode) == 0
