@@ -65,7 +65,7 @@ extern "C" {
 #define BCAST_SHAPE_AUTO     (-1)       /* chosen per call from an estimate (the default)          */
 #define BCAST_SHAPE_BLOCK      0        /* a block per tile, undecided entries searched per tile   */
 #define BCAST_SHAPE_WARPS      1        /* warps on their own, searches deferred to the block's end */
-#define BCAST_SHAPE_LOWFRAME   2        /* the same, low rounds looked up in a per-block table     */
+#define BCAST_SHAPE_LOWFRAME   2        /* the same, low rounds looked up in a table of low states */
 #define BCAST_SHAPE_WARPS_TIGHT 3       /* BCAST_SHAPE_WARPS with next to no queue space: for tests */
                                         /* of the path that recomputes a group whose queues ran full */
 

@@ -303,8 +303,8 @@ static std::atomic<int> &forced_shape()
 
 // Which launch shape suits p.  With next to no undecided entries (at most 0.05 of Algorithm 6's
 // violations per rank; p = 2^27-1 has none) the warps go through the tiles on their own and the block
-// runs the few searches at the end.  With more, each block first tabulates the low rounds of the
-// search for every low state (low_frame_entry), which settles most undecided entries by a lookup and
+// runs the few searches at the end.  With more, the launch carries the low rounds of the search
+// tabulated for every low state (low_frame_fill), which settles most undecided entries by a lookup and
 // leaves few enough searches for the same shape.  The block-per-tile shape, which meets after every
 // tile and drains its queues there, serves the shifted tables, small q and descending rows below
 // kDescWarpsFromQ.  A wrong estimate costs time, never correctness.
@@ -331,15 +331,16 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     const LevelTables tab = host_tables(p, q);
     const int shape = choose_shape(tab, p, q, descending, shift_x);
     // up to kWarpsPerBlock consecutive tiles per block, fewer while the grid would have less than
-    // kBlocksPerSmWanted blocks per SM (short launches want many small blocks).  A block that first
-    // tabulates the search's low states takes more tiles to spread that cost: up to kLowFrameTiles.
+    // kBlocksPerSmWanted blocks per SM (short launches want many small blocks).  A block that works with
+    // the table of the search's low states copies it to shared memory first and gathers its deferred
+    // searches over several groups of tiles, so it takes more: up to kLowFrameTiles.
     int64_t tiles_per_block = n_tiles / ((int64_t)sms * kBlocksPerSmWanted);
     if (tiles_per_block < 1) tiles_per_block = 1;
     if (tiles_per_block > kWarpsPerBlock) tiles_per_block = kWarpsPerBlock;
     if (shape == kShapeWarpsLowFrame) {
-        // one wave of resident blocks while that keeps a block within kLowFrameTiles tiles (measured best
-        // from p = 2^20+1 to 2^24+3), else blocks of kLowFrameTiles (p = 1.2e8: 64 or 128 tiles alike,
-        // fewer is slower)
+        // one wave of resident blocks while that keeps a block within kLowFrameTiles tiles, else blocks of
+        // kLowFrameTiles (measured: p = 2^20+1 best at 4 tiles, 2^22+1 at 8 to 16, 2^24+3 and 1.2e8 at 16
+        // to 32; fewer than 4 or more than 32 is slower everywhere)
         const int64_t slots = (int64_t)sms * kTableBlocksPerSm;
         tiles_per_block = (n_tiles + slots - 1) / slots;
         if (tiles_per_block > kLowFrameTiles) tiles_per_block = kLowFrameTiles;
@@ -361,6 +362,14 @@ static int launch_table(int32_t p, int q, int32_t anchor, int64_t row_begin, int
     launch.send_vec = send_vec;
     launch.shift_x = shift_x;
     launch.shape = shape;
+    memset(&launch.low_states, 0xff, sizeof(launch.low_states));
+    if (shape == kShapeWarpsLowFrame) {
+        Geometry g;
+        g.p = (uint32_t)p;
+        g.pm1 = (uint32_t)p - 1u;
+        g.q = q;
+        low_frame_fill(g, kSharedFrom, launch.low_states.word, (uint32_t)kLowFrameStates);
+    }
     launch.grid = grid;
     launch.stream = (cudaStream_t)cuda_stream;
     if (!(launch_table_q_low(launch, q) || launch_table_q_mid(launch, q) || launch_table_q_high(launch, q) ||

@@ -43,9 +43,19 @@ __device__ __forceinline__ Geometry make_geometry(uint32_t p)
 }
 
 // Algorithm 2 in closed form; valid for 0 <= k <= q.
-__device__ __forceinline__ uint32_t skip_of(const Geometry &g, int k)
+__host__ __device__ __forceinline__ uint32_t skip_of(const Geometry &g, int k)
 {
     return (g.pm1 >> (g.q - k)) + 1u;
+}
+
+// Index of the highest set bit of x != 0.
+__host__ __device__ __forceinline__ int top_bit(uint32_t x)
+{
+#ifdef __CUDA_ARCH__
+    return 31 - __clz(x);
+#else
+    return 31 - __builtin_clz(x);
+#endif
 }
 
 // Algorithm 3: smallest index of the canonical skip sequence of r; q for r = 0.
@@ -69,12 +79,12 @@ struct SearchStats {
 };
 
 struct NoStats {
-    __device__ __forceinline__ void begin() {}
-    __device__ __forceinline__ void descent() {}
-    __device__ __forceinline__ void step() {}
-    __device__ __forceinline__ void cap() {}
-    __device__ __forceinline__ void end(int) {}
-    __device__ __forceinline__ void violation(uint32_t, int) {}
+    __host__ __device__ __forceinline__ void begin() {}
+    __host__ __device__ __forceinline__ void descent() {}
+    __host__ __device__ __forceinline__ void step() {}
+    __host__ __device__ __forceinline__ void cap() {}
+    __host__ __device__ __forceinline__ void end(int) {}
+    __host__ __device__ __forceinline__ void violation(uint32_t, int) {}
 };
 
 struct CountStats {
@@ -162,7 +172,7 @@ __device__ __forceinline__ SearchState search_from_digits(const Geometry &g, uin
 // value (b where the search accepted index q, else index - q).  k_last = q-1 yields
 // the whole row; a smaller k_last stops early.
 template <class Emit, class Stats>
-__device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchState &st, int k_last,
+__host__ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchState &st, int k_last,
                                                 Emit emit, Stats &stats)
 {
     const int q = g.q;
@@ -175,7 +185,7 @@ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchS
     int k = st.k;
     uint32_t sk_k = skip_of(g, k);                        // skip[k]
     uint32_t sk_k1 = skip_of(g, k + 1 <= q ? k + 1 : q);  // skip[k+1]
-    uint32_t m = max(sk_k, v + 1u);                       // max(skip[k], v+1)
+    uint32_t m = sk_k > v + 1u ? sk_k : v + 1u;           // max(skip[k], v+1)
     int guard = 6 * q + 16;                               // never reached; keeps the loop finite
 
     while (true) {
@@ -188,7 +198,7 @@ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchS
         uint32_t bit, sk_e;
         bool accept;
         if (cand != 0u) {
-            e = 31 - __clz(cand);
+            e = top_bit(cand);
             bit = 1u << e;
             cand ^= bit;
             sk_e = skip_of(g, e);
@@ -207,7 +217,7 @@ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchS
             if (pending == 0u) { stats.end(q); return; }  // outermost call ran off the list
             bit = pending & (0u - pending);               // innermost pending call
             pending ^= bit;
-            e = 31 - __clz(bit);
+            e = top_bit(bit);
             sk_e = skip_of(g, e);
             u += sk_e;                                    // back in the caller's frame
             accept = (u >= sk_k1);                        // else the caller returns as well
@@ -221,7 +231,7 @@ __device__ __forceinline__ void recv_search_run(const Geometry &g, const SearchS
             ++k;
             sk_k = sk_k1;
             sk_k1 = skip_of(g, k + 1 <= q ? k + 1 : q);
-            m = max(sk_k, v + 1u);
+            m = sk_k > v + 1u ? sk_k : v + 1u;
         }
     }
 }
@@ -312,16 +322,16 @@ __device__ __forceinline__ int recv_entry(const Geometry &g, uint32_t t, int k, 
 // down, so its first rounds are the entry of u'; where that stretch ends it returns to x
 // and accepts it.  (u' = 1: x is accepted for round 0 at once.  u' = 0: x is the baseblock
 // and not in the list.)  Only what follows needs the search itself, started from the state
-// that prefix leaves: back in the outermost call, scanning below x.  A block fills the
-// table level by level (all u with the same highest digit side by side, a barrier between
-// the levels).
+// that prefix leaves: back in the outermost call, scanning below x.  The table depends on
+// p alone, so the host fills it once per launch, in increasing u (low_frame_fill), and
+// hands it to the kernel among its arguments; every block copies it to shared memory.
 constexpr uint32_t kLowFramePop = 14u;
 constexpr uint32_t kLowFrameNone = 15u;
 constexpr int kLowFrameRounds = 8;
 
 // Entry of u, skip[x] <= u < skip[x+1], given the entries of every smaller u.
-__device__ __forceinline__ uint32_t low_frame_entry(const Geometry &g, int L, const uint32_t *table, int x,
-                                                    uint32_t u)
+__host__ __device__ __forceinline__ uint32_t low_frame_entry(const Geometry &g, int L, const uint32_t *table,
+                                                             int x, uint32_t u)
 {
     constexpr uint32_t kNone = 0xffffffffu;
     if (u < 2u) return kNone;
@@ -374,15 +384,15 @@ __device__ __forceinline__ uint32_t low_frame_entry(const Geometry &g, int L, co
     return packed;
 }
 
-// Fills table[0 .. min(skip[L], capacity)) ; called by every thread of the block.
-__device__ __forceinline__ void low_frame_build(const Geometry &g, int L, uint32_t *table, uint32_t capacity)
+// Fills table[0 .. min(skip[L], capacity)), every entry from the ones before it.
+inline void low_frame_fill(const Geometry &g, int L, uint32_t *table, uint32_t capacity)
 {
-    const uint32_t n_states = min(skip_of(g, L), capacity);
-    if (threadIdx.x < 2u) table[threadIdx.x] = 0xffffffffu;
+    const uint32_t n_states = skip_of(g, L) < capacity ? skip_of(g, L) : capacity;
+    for (uint32_t u = 0; u < 2u && u < n_states; ++u) table[u] = 0xffffffffu;
     for (int x = 1; x < L; ++x) {
-        const uint32_t lo = skip_of(g, x), hi = min(skip_of(g, x + 1), n_states);
-        for (uint32_t u = lo + threadIdx.x; u < hi; u += blockDim.x) table[u] = low_frame_entry(g, L, table, x, u);
-        __syncthreads();
+        const uint32_t lo = skip_of(g, x);
+        const uint32_t hi = skip_of(g, x + 1) < n_states ? skip_of(g, x + 1) : n_states;
+        for (uint32_t u = lo; u < hi; ++u) table[u] = low_frame_entry(g, L, table, x, u);
     }
 }
 

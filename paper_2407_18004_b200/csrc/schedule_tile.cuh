@@ -385,8 +385,13 @@ struct DeferredItem {
 constexpr int kDeferredCapacity = 384;
 constexpr int kFixupCapacity = 768;
 constexpr int kGroupRows = kWarpsPerBlock * kThreads;  // rows of a group of tiles
-constexpr int kLowFrameTiles = 64;                     // most tiles of a block that builds the table of low states
+constexpr int kLowFrameTiles = 16;                     // most tiles of a block that works with the table of low states
 constexpr int kLowFrameStates = 512;                   // skip[kSharedFrom] <= 2^kSharedFrom states of the low frame
+
+// The table of low states as the host hands it to the kernel (low_frame_fill).
+struct LowFrameTable {
+    uint32_t word[kLowFrameStates];
+};
 
 // Launch shapes of the table kernel.
 constexpr int kShapeBlockPerTile = 0;                  // the block meets after every tile and drains its queues
@@ -399,7 +404,7 @@ constexpr int kDescWarpsFromQ = 16;                    // smallest q with a desc
 struct DeferredQueue {
     DeferredItem items[kDeferredCapacity];
     uint32_t fixups[kFixupCapacity];                       // row relative to the block | k << 14
-    uint32_t low_frame[kLowFrameStates];                   // low_frame_entry(u) for u < skip[kSharedFrom], if built
+    uint32_t low_frame[kLowFrameStates];                   // low_frame_entry(u) for u < skip[kSharedFrom], if given
     uint32_t need_recv[kWarpsPerBlock][32];                // per warp and row of its slice: rounds to search
     int n_items;
     int n_fixups;

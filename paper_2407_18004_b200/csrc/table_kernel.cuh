@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(kThreads, kTableBlocksPerSm)
 schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint32_t anchor,
                       uint32_t row_begin, uint32_t n_ranks, int descending, int tiles_per_block,
                       int32_t *__restrict__ recv_out, int32_t *__restrict__ send_out,
-                      int recv_vec_ok, int send_vec_ok, int shift_x, int shape)
+                      int recv_vec_ok, int send_vec_ok, int shift_x, int shape,
+                      const __grid_constant__ LowFrameTable low_states)
 {
     typedef typename WalkInt<Q>::type Int;
     __shared__ uint32_t stage[2][(kThreads * Q + 15) / 16 * 4];   // byte tiles, kThreads rows of Q entries
@@ -68,13 +69,13 @@ schedule_table_kernel(const __grid_constant__ LevelTables tab, uint32_t p, uint3
         DeferredQueue &dq = queues.deferred;
         if (threadIdx.x == 0) { dq.n_items = 0; dq.n_fixups = 0; }
         if (threadIdx.x == 2) dq.overflow = 0u;
-        // the low rounds of the search for every low state of this p, when the host expects
-        // enough undecided entries to pay for it
+        // the low rounds of the search for every low state of this p, filled in by the host when it
+        // expects enough undecided entries to pay for the lookups
         const int capacity_cut = shape == kShapeWarpsTight ? kDeferredCapacity - kTightCapacity : 0;
         const uint32_t *low_frame = nullptr;
         if constexpr (Q >= kSharedFrom + 2) {
             if (shape == kShapeWarpsLowFrame) {            // the same for the whole block
-                low_frame_build(g, kSharedFrom, dq.low_frame, (uint32_t)kLowFrameStates);
+                for (int i = threadIdx.x; i < kLowFrameStates; i += kThreads) dq.low_frame[i] = low_states.word[i];
                 low_frame = dq.low_frame;
             }
         }
@@ -194,6 +195,7 @@ struct TableLaunch {
     int32_t *recv_dev, *send_dev;
     int recv_vec, send_vec, shift_x;
     int shape;                          // kShape*; descending rows take a warps shape only for q >= kDescWarpsFromQ
+    LowFrameTable low_states;           // filled for kShapeWarpsLowFrame only
 
     int grid;
     cudaStream_t stream;
@@ -206,13 +208,13 @@ static void launch_table_kernel(const TableLaunch &l)
         if (l.descending && l.shape != kShapeBlockPerTile) {
             schedule_table_kernel<N, true><<<l.grid, kThreads, 0, l.stream>>>(
                 l.tab, l.p, l.anchor, l.row_begin, l.n_rows, l.descending, l.tiles_per_block, l.recv_dev,
-                l.send_dev, l.recv_vec, l.send_vec, l.shift_x, l.shape);
+                l.send_dev, l.recv_vec, l.send_vec, l.shift_x, l.shape, l.low_states);
             return;
         }
     }
     schedule_table_kernel<N, false><<<l.grid, kThreads, 0, l.stream>>>(
         l.tab, l.p, l.anchor, l.row_begin, l.n_rows, l.descending, l.tiles_per_block, l.recv_dev, l.send_dev,
-        l.recv_vec, l.send_vec, l.shift_x, l.descending ? kShapeBlockPerTile : l.shape);
+        l.recv_vec, l.send_vec, l.shift_x, l.descending ? kShapeBlockPerTile : l.shape, l.low_states);
 }
 
 // One translation unit per range of q (they compile side by side); each returns false for
