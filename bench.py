@@ -484,9 +484,18 @@ def measure_configs(bs, torch, recv, send, stream, peak, headline_ms, p_large):
         mean_ms, min_ms = time_launches(torch, stream, fn, pairs, per_pair)
         nbytes = 8 * q * p
         gbs = nbytes / (mean_ms * 1e-3) / 1e9
+        # the store pattern alone over the same two tables, launched the same way: what a launch of this size can reach
+        def fill():
+            bs.bcast_store_ceiling(r, r.numel() * 4, 0, stream)
+            bs.bcast_store_ceiling(s_, s_.numel() * 4, 0, stream)
+        fill()
+        torch.cuda.synchronize()
+        fill_ms, _ = time_launches(torch, stream, fill, 3, per_pair)
+        store_gbs = nbytes / (fill_ms * 1e-3) / 1e9
         out[name] = {"workload": what % (p, q), "ms": mean_ms, "ms_min": min_ms, "launches_per_event_pair": per_pair,
                      "value": p / (mean_ms * 1e-3), "unit": UNIT, "bytes_per_launch": nbytes,
-                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak}}
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                  "store_only_gbs": store_gbs, "frac_of_store_only": gbs / store_gbs}}
         return mean_ms
 
     table_entry("config2_p=2^20+1", workloads.P_MEDIUM,
