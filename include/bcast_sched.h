@@ -418,6 +418,27 @@ int bcast_simulate_allreduce(int32_t p, int64_t n,
 int bcast_store_ceiling(void *buffer_dev, int64_t bytes, int64_t bytes_per_block, void *cuda_stream);
 
 /*
+ * The table of the search's low states that bcast_schedule hands to its kernel
+ * for p whose closed forms leave many entries undecided (no counterpart in the
+ * paper as a table: it is Algorithms 4 and 5 memoised on the search's state).
+ * Let u be what is left of p + r after the greedy digits of p + r over the
+ * skips at the levels >= BCAST_LOW_LEVELS (skip[q] = p first).  For u >= 2 the
+ * first rounds of the receive schedule of virtual rank r depend on u alone:
+ * nibble k (bits 4k..4k+3, k = 0..7) of states_host[u] is the skip index e the
+ * search accepts in round k, i.e. recvblock[k] = e - q; 14 where the search
+ * returns past the low levels and accepts the lowest digit j >= BCAST_LOW_LEVELS
+ * of p + r (recvblock[k] = j - q, or the baseblock of r when j = q); 15 for the
+ * rounds after that one, which the table does not hold.  Entries 0 and 1 are
+ * all-ones.  Fills min(skip[BCAST_LOW_LEVELS], capacity) words of states_host
+ * (host memory, capacity >= 0) and returns that count; 0 for q < BCAST_LOW_LEVELS + 2,
+ * where the kernels do not use it.
+ * Pure host computation, no CUDA call.  Errors: BCAST_EINVAL_P, BCAST_ENULL,
+ * BCAST_EINVAL_N (capacity < 0).
+ */
+#define BCAST_LOW_LEVELS 9
+int bcast_low_states(int32_t p, uint32_t *states_host, int32_t capacity);
+
+/*
  * Algorithm 1's use of a schedule row, O(1) per round.  For n >= 1 blocks and
  * communication round j in [0, n-1+q): x = (q - (n-1) mod q) mod q virtual
  * rounds come first, so i = x + j, k = i mod q is the skip index of the round

@@ -57,6 +57,7 @@ def _load():
         lib.bcast_simulate_broadcast.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_simulate_reduce.argtypes = [i32, i32, i64, vp, vp, vp, vp, vp, vp, i64, vp]
         lib.bcast_store_ceiling.argtypes = [vp, i64, i64, vp]
+        lib.bcast_low_states.argtypes = [i32, vp, i32]
         lib.bcast_simulate_all_scratch_bytes.argtypes = [i32, i64, ctypes.c_int]
         lib.bcast_simulate_all_scratch_bytes.restype = i64
         lib.bcast_simulate_allbroadcast.argtypes = [i32, i64, vp, vp, vp, vp, vp, i64, vp]
@@ -121,6 +122,12 @@ def bcast_skips(p: int) -> np.ndarray:
 
 def bcast_store_ceiling(buffer, nbytes: int, bytes_per_block: int = 0, stream=None) -> int:
     return _check(_load().bcast_store_ceiling(_ptr(buffer), nbytes, bytes_per_block, _stream(stream)))
+
+
+def bcast_low_states(p: int, capacity: int = 512) -> np.ndarray:
+    out = np.zeros(capacity, dtype=np.uint32)
+    count = _check(_load().bcast_low_states(p, out.ctypes.data, capacity))
+    return out[:count]
 
 
 def bcast_round(q: int, n: int, j: int):

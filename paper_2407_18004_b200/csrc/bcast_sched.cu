@@ -513,6 +513,23 @@ int bcast_store_ceiling(void *buffer_dev, int64_t bytes, int64_t bytes_per_block
     return BCAST_OK;
 }
 
+int bcast_low_states(int32_t p, uint32_t *states_host, int32_t capacity)
+{
+    static_assert(BCAST_LOW_LEVELS == kSharedFrom, "public and internal number of low levels agree");
+    if (p < 1) return BCAST_EINVAL_P;
+    if (states_host == nullptr) return BCAST_ENULL;
+    if (capacity < 0) return BCAST_EINVAL_N;
+    const int q = host_q(p);
+    if (q < kSharedFrom + 2) return 0;
+    Geometry g;
+    g.p = (uint32_t)p;
+    g.pm1 = (uint32_t)p - 1u;
+    g.q = q;
+    low_frame_fill(g, kSharedFrom, states_host, (uint32_t)capacity);
+    const uint32_t states = skip_of(g, kSharedFrom);
+    return (int)(states < (uint32_t)capacity ? states : (uint32_t)capacity);
+}
+
 int bcast_round(int32_t q, int64_t n, int64_t j, int32_t *k_out, int64_t *shift_out)
 {
     if (q < 1 || n < 1) return BCAST_EINVAL_N;

@@ -136,3 +136,59 @@ def test_workload_generator_is_seeded_and_in_range():
     # log-uniform: every octave between 2^1 and 2^31 is populated
     octave = np.floor(np.log2(p.astype(np.float64))).astype(int)
     assert set(range(1, 31)) <= set(octave.tolist())
+
+
+def test_low_state_table_matches_oracle_receive_schedules():
+    """The table of the search's low states, which the host fills and the table kernel looks undecided low rounds
+    up in: every state's rounds against the oracle's receive schedule (Algorithm 5) of ranks in that state."""
+    levels = 9
+    rng = np.random.default_rng(11)
+    ps = [2 ** 11 + 1, 3000, 2 ** 12 - 1, 40001, 2 ** 16 + 1, 2 ** 20 + 1, 3858024, 2 ** 24 + 3, 123456789,
+          2 ** 27 - 1, 2 ** 31 - 1]
+    assert len(bs.bcast_low_states(1000)) == 0 and len(bs.bcast_low_states(1024)) == 0      # q = 10: not used
+    for p in ps:
+        q = oracle.q_of(p)
+        skip = [int(x) for x in oracle.skips(p)]
+        states = bs.bcast_low_states(p)
+        assert len(states) == skip[levels] and states[0] == states[1] == 0xFFFFFFFF
+        assert list(bs.bcast_low_states(p, 100)) == list(states[:100])
+        ranks = range(1, p) if p <= 5000 else [int(x) for x in rng.integers(1, p, 1500)]
+        seen = set()
+        for r in ranks:
+            # what is left of p + r after its greedy digits at the levels >= 9 (skip[q] = p comes first, leaving r)
+            u, j = r, q
+            for k in range(q - 1, levels - 1, -1):
+                if u >= skip[k]:
+                    u -= skip[k]
+                    j = k
+            if u < 2:
+                continue
+            seen.add(u)
+            recv = oracle.recvschedule(p, r)
+            popped = oracle.baseblock(p, r) if j == q else j - q
+            word = int(states[u])
+            rounds = 0
+            for k in range(8):
+                nib = (word >> (4 * k)) & 15
+                if nib == 15:
+                    break
+                assert int(recv[k]) == (popped if nib == 14 else nib - q), (p, r, u, k, hex(word))
+                rounds += 1
+                if nib == 14:
+                    assert all((word >> (4 * kk)) & 15 == 15 for kk in range(k + 1, 8)), (p, u, hex(word))
+                    break
+            else:
+                assert int(recv[8]) == popped, (p, r, u, hex(word))        # eight rounds used up every low index
+            assert rounds >= 1, (p, r, u, hex(word))
+        assert len(seen) >= min(200, skip[levels] - 2) or p > 5000, (p, len(seen))
+
+
+def test_low_state_table_argument_errors():
+    buf = np.zeros(8, dtype=np.uint32)
+    lib = ctypes.CDLL(bs.library_path())
+    lib.bcast_low_states.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32]
+    assert lib.bcast_low_states(0, buf.ctypes.data, 8) == -1
+    assert lib.bcast_low_states(5000, None, 8) < 0
+    assert lib.bcast_low_states(5000, buf.ctypes.data, -1) < 0
+    assert lib.bcast_low_states(5000, buf.ctypes.data, 8) == 8
+    assert lib.bcast_low_states(5000, buf.ctypes.data, 0) == 0
