@@ -6,7 +6,9 @@ back as int8 and compared element by element.
 
   config 3  every receive row of p = 2^27-1 (134 217 727 rows; about two minutes of one core), and then
             condition 2 over the whole device tables, which with a verified receive table IS the
-            definition of the send table (Section 2.3);
+            definition of the send table (Section 2.3); the same for p = 123 456 789 with root
+            floor(p/3), a p whose closed forms leave entries undecided, and for p = 2^26+1 (every
+            skip odd), root 12345;
   config 4  the checksum of every p in [2, 65536] against tests/golden/checksums_2_65536.txt, which
             tests/golden/make_checksums.py wrote from the oracle;
   config 5  every receive row of the 2^24 queries against Algorithm 5 and every send row against the
@@ -40,17 +42,21 @@ def first_difference(name, got, want, lo):
         name, len(bad), lo + r, k, got[r, k], want[r, k])
 
 
-def test_config3_every_receive_row_and_the_send_table_by_definition():
-    p = workloads.P_LARGE
+@pytest.mark.parametrize("p, root", [(workloads.P_LARGE, 0), (123456789, 123456789 // 3), (2 ** 26 + 1, 12345)],
+                         ids=["config3_p=2^27-1_root0", "ordinary_p=123456789_root_p/3", "odd_skips_p=2^26+1_root12345"])
+def test_config3_every_receive_row_and_the_send_table_by_definition(p, root):
+    # the second case is a p with no special form (0.3 of Algorithm 6's violations per rank: lookups in the
+    # table of low states, deferred searches gathered over groups of tiles, fix-ups) and a root other than 0;
+    # the third has every skip odd (1.5 violations per rank, the densest queues) at q = 27
     q = bs.bcast_q(p)
     free, _ = torch.cuda.mem_get_info()
     if free < 34 * 2 ** 30:
         pytest.skip("needs 34 GB of device memory")
     oracle.build()
-    recv, send = bs.schedule(p)
+    recv, send = bs.schedule(p, root)
     torch.cuda.synchronize()
     chunk = 2 ** 22
-    jobs = [(p, 0, lo, min(p, lo + chunk)) for lo in range(0, p, chunk)]
+    jobs = [(p, root, lo, min(p, lo + chunk)) for lo in range(0, p, chunk)]
     with mp.get_context("spawn").Pool(oracle_workers.pool_size()) as pool:
         for (_, _, lo, hi), want in zip(jobs, pool.imap(oracle_workers.recv_rows, jobs)):
             got = recv[lo:hi].to(torch.int8).cpu().numpy()
