@@ -202,6 +202,8 @@ struct TileRuns {
     uint32_t level[kMaxRuns][kSharedLevels];   // send entry | receive entry before the switch << 8 | switch offset << 16;
                                                // from the switch on the receive entry is k - q
     uint32_t pending[kMaxPending];          // row | k << 9 | is_send << 14
+    uint32_t full_len[kMaxRuns];            // ranks from the run's first row on that share its digits and lie below p,
+                                            // also past the tile's end
 };
 
 // Executed by one whole warp.  tab: uniform-index tables; lookup: tables for per-lane indices.
@@ -247,10 +249,11 @@ __device__ __forceinline__ void build_tile_runs(const LevelTables &tab, const Le
         if (my == kSharedFrom - 1) { my_rp = rem; my_e = e; }
         const bool upper = column && ((digits >> k) & 1u);
         // the run ends where a clear digit's remainder reaches its skip
-        Int run = column && !upper ? sk - my_rp : (Int)rows;
+        Int run = column && !upper ? sk - my_rp : (Int)0x7fffffff;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) run = min(run, __shfl_xor_sync(kFull, run, off));
         const int n = (int)min(run, (Int)(rows - ib));          // rows ib .. ib+n-1
+        if (lane == 0) out.full_len[n_runs] = (uint32_t)min(run, (Int)p - (Int)base);
 
         // ---- step 2: what level `my` sees above it
         const uint32_t above = owner ? digits >> (my + 1) : 0u;

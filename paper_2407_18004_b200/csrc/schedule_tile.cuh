@@ -487,10 +487,11 @@ __device__ __forceinline__ uint32_t low_frame_values(uint32_t word, int j_high, 
 // Undecided low rounds from the table of the search's low states (low_frame_entry): the
 // rank's own receive entries from its own state u_low, and its send entries from the state
 // of its to-processor where that is a rank of the same run (same digits at the levels
-// >= kSharedFrom, u_low + skip[k] left below them).
+// >= kSharedFrom, u_low + skip[k] left below them), whether or not it is a row of the same
+// tile: `room` = the ranks from this one on that lie in its run and below p.
 template <int Q, class Row>
 __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const uint32_t *low_frame,
-                                                  uint32_t u_low, int j_high, uint32_t ahead, uint32_t run_end,
+                                                  uint32_t u_low, int j_high, uint32_t room,
                                                   Row recv_row, Row send_row, uint32_t &recv_flags,
                                                   uint32_t &send_flags, bool any_recv)
 {
@@ -512,7 +513,7 @@ __device__ __forceinline__ void low_frame_lookups(const LevelTables &tab, const 
         const int k = __ffs(todo) - 1;
         todo &= todo - 1u;
         const uint32_t skip_k = skip_of(make_geometry(tab.skip[Q]), k);
-        if (ahead + skip_k < run_end) {
+        if (skip_k < room) {
             const uint32_t word_t = low_frame[u_low + skip_k];
             const uint32_t nib = k < kLowFrameRounds ? (word_t >> (4 * k)) & 15u
                                                      : (low_frame_full(word_t) ? kLowFramePop : kLowFrameNone);
@@ -602,11 +603,12 @@ __device__ __forceinline__ void warp_pass(const LevelTables &tab, const Geometry
                 int run = 0;
 #pragma unroll
                 for (int i = 1; i < kMaxRuns; ++i) run += (int)ahead >= runs.start[i] ? 1 : 0;
-                const uint32_t u_low = (uint32_t)runs.state[run].rp + (ahead - (uint32_t)runs.start[run]);
+                const uint32_t t = ahead - (uint32_t)runs.start[run];
+                const uint32_t u_low = (uint32_t)runs.state[run].rp + t;
                 const int j_high = runs.state[run].j;      // lowest digit at the shared levels (Q: none)
                 const bool any_recv = __any_sync(0xffffffffu, (recv_flags & kLowMask) != 0u);
                 if (j_high < Q)
-                    low_frame_lookups<Q>(tab, low_frame, u_low, j_high, ahead, (uint32_t)runs.start[run + 1],
+                    low_frame_lookups<Q>(tab, low_frame, u_low, j_high, runs.full_len[run] - t,
                                          recv_row, send_row, recv_flags, send_flags, any_recv);
             }
             // entries of the high levels that the description left undecided (at most 32, one per
